@@ -1,0 +1,147 @@
+/*
+ * ziplm.h -- C ABI of the layer-wise structured Optimal-Brain-Surgeon solver of ZipLM
+ * (arXiv 2302.04089, Sec. 3.1, Algorithm 1) for NVIDIA B200 (sm_100a).
+ *
+ * Conventions shared by every entry point
+ *   - "dev" pointers are CUDA device pointers of the current device, "host" pointers are
+ *     ordinary host memory.  All matrices are dense row-major.
+ *   - The caller owns every buffer.  The library allocates no device memory, creates no stream
+ *     and keeps no state between calls.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = the default
+ *     stream) and the call returns without synchronising.  Buffers must stay alive until the
+ *     stream has drained.
+ *   - The return value reports what the host can see when the work is enqueued (bad arguments,
+ *     workspace too small, a failed launch).  Failures that depend on the data (a Hessian that
+ *     is not positive definite, non-finite values) are written to `layer_status[l]` on the
+ *     device; the outputs of such a layer are unspecified but in bounds and the other layers
+ *     are unaffected.
+ *   - There is no CPU fallback: without a CUDA device the compute entry points return
+ *     ZIPLM_ERR_CUDA.
+ *
+ * Notation (the paper's): W is d_row x d_col, X is d_col x n_tokens (one calibration token per
+ * column), H = 2 X X^T, a structure is `group_size` consecutive columns of W (1 = FFN neuron,
+ * 64 = attention head), G = d_col / group_size structures per layer, L same-shape layers are
+ * processed together because the method treats every layer independently (Sec. 3.2).
+ */
+#ifndef ZIPLM_H_
+#define ZIPLM_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ZIPLM_OK = 0,
+    ZIPLM_ERR_INVALID_ARG = 1, /* shape, pointer or level list rejected on the host            */
+    ZIPLM_ERR_WORKSPACE = 2,   /* workspace pointer NULL / misaligned / smaller than required  */
+    ZIPLM_ERR_NOT_PD = 3,      /* damped Hessian not positive definite (per layer)             */
+    ZIPLM_ERR_NONFINITE = 4,   /* NaN or Inf met in H, W or a saliency (per layer)             */
+    ZIPLM_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out                           */
+    ZIPLM_ERR_CUDA = 6,        /* a CUDA runtime call or kernel launch failed                  */
+    ZIPLM_ERR_UNSUPPORTED = 7  /* valid request outside what this build implements            */
+} ziplm_status;
+
+typedef enum { ZIPLM_F32 = 0, ZIPLM_BF16 = 1 } ziplm_dtype;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* ziplm_status_string(ziplm_status s);
+
+/* ---------------------------------------------------------------------------------------------
+ * Calibration Hessian (caption of Algorithm 1: H = 2 X X^T; "Saliency scores and weight update").
+ *
+ *   H[l] = beta * H[l] + alpha * X[l] X[l]^T        for l = 0 .. L-1
+ *
+ * alpha = 2 gives the paper's Hessian; beta = 1 adds one more batch of tokens to a running sum,
+ * beta = 0 overwrites.  Products are accumulated in fp32; fp32 inputs keep fp32 accuracy (on the
+ * tensor-core route they are split into TF32 terms), bf16 inputs are multiplied exactly.
+ *
+ *   H          dev, [L, d, d] fp32, in/out; full symmetric matrix on return
+ *   X          dev, [L, d, ldx] of x_dtype, token index contiguous; only the first n_tokens
+ *              entries of each row are read; not modified.  The base address must be 16-byte
+ *              aligned and ldx * sizeof(element) a multiple of 16.
+ *   ldx        row pitch of X in elements, >= n_tokens
+ *   workspace  dev scratch of at least ziplm_hessian_workspace_bytes(...) bytes, 256-byte
+ *              aligned; may be NULL when that size is 0
+ *
+ * Errors: ZIPLM_ERR_INVALID_ARG for L, d < 1, n_tokens < 0, ldx < n_tokens, a NULL pointer,
+ * misaligned X or beta outside {0, 1}; ZIPLM_ERR_WORKSPACE; ZIPLM_ERR_CUDA.
+ * n_tokens = 0 scales H by beta and returns.
+ */
+size_t ziplm_hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype x_dtype);
+
+ziplm_status ziplm_hessian_accumulate(float* H, const void* X, ziplm_dtype x_dtype, int L, int d,
+                                      long long n_tokens, long long ldx, float alpha, float beta,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Damped inverse (caption of Algorithm 1: H^-1 = (2 X X^T + lambda I)^-1).
+ *
+ *   lambda[l] = damp_frac * mean(diag H[l]);   Hinv[l] = (H[l] + lambda[l] I)^-1
+ *
+ * computed in float64 through a blocked Cholesky factorisation H + lambda I = C C^T, the inverse
+ * of the triangular factor and the product C^-T C^-1.  This is the first stage of
+ * ziplm_prune_layers, exported so that it can be used and checked on its own.
+ *
+ *   H             dev, [L, d, d] fp32, symmetric (only the lower triangle is read); not modified
+ *   Hinv          dev, [L, d, d] fp64, full symmetric matrix on return
+ *   layer_status  dev, [L] int: ZIPLM_OK, ZIPLM_ERR_NOT_PD (a pivot <= 0 or mean(diag) <= 0
+ *                 with damp_frac > 0) or ZIPLM_ERR_NONFINITE
+ *   workspace     dev scratch >= ziplm_inverse_workspace_bytes(L, d), 256-byte aligned
+ */
+size_t ziplm_inverse_workspace_bytes(int L, int d);
+
+ziplm_status ziplm_damped_inverse(const float* H, int L, int d, float damp_frac, double* Hinv,
+                                  int* layer_status, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Greedy structured pruning of L same-shape layers (Algorithm 1; Eq. 2, Eq. 3, Eq. 4) with a
+ * snapshot at every requested level (the per-layer database of Sec. 3.2).
+ *
+ * For every layer: dampen and invert H as above; then, until min(levels) structures remain,
+ * score every remaining structure S with
+ *     rho_S = sum_i W[i,S] ((H^-1)[S,S])^-1 W[i,S]^T                           (Eq. 2)
+ * remove the structure with the smallest rho (ties: lowest structure index), apply
+ *     W <- W - W[:,S] ((H^-1)[S,S])^-1 (H^-1)[S,:]                             (Eq. 3)
+ *     H^-1 <- H^-1 - (H^-1)[:,S] ((H^-1)[S,S])^-1 (H^-1)[S,:]                  (Eq. 4)
+ * and, whenever the number of remaining structures equals an entry of `levels`, store the
+ * weights with the removed columns set to exactly zero (last line of Algorithm 1) together with
+ * the reconstruction loss of Eq. 1.
+ *
+ *   W            dev, [L, d_row, d_col] fp32; not modified
+ *   H            dev, [L, d_col, d_col] fp32, the UNDAMPED 2 X X^T, symmetric; not modified
+ *   group_size   columns per structure; d_col % group_size == 0; 1 <= group_size <= 64
+ *   damp_frac    lambda = damp_frac * mean(diag H[l]); >= 0
+ *   levels       HOST, [n_levels] numbers of REMAINING structures, strictly decreasing, each in
+ *                [0, G]; level 0 removes the whole module, level G is the unpruned layer
+ *   W_snap       dev, [L, n_levels, d_row, d_col] fp32
+ *   loss         dev, [L, n_levels] fp32:  ||(W - W_snap) X||_F^2  (no damping term)
+ *   base_loss    dev, [L] fp32:  ||W X||_F^2 ; may be NULL
+ *   order        dev, [L, G] int: structure removed at step t, -1 for steps that did not run
+ *   saliency     dev, [L, G] fp32: rho of the structure removed at step t (0 past the end);
+ *                may be NULL
+ *   layer_status dev, [L] int, per-layer ziplm_status
+ *   workspace    dev scratch >= ziplm_prune_workspace_bytes(...), 256-byte aligned
+ *
+ * The loss is evaluated through the identity  loss + lambda/2 ||W - W_snap||_F^2 = 1/2 * (sum of
+ * the rho of the structures removed so far), which holds because every rho is twice the increase
+ * of the damped least-squares objective; it needs no extra pass over H.
+ *
+ * Errors: ZIPLM_ERR_INVALID_ARG (shapes, NULL pointers, levels not strictly decreasing or out
+ * of range, damp_frac < 0 or not finite), ZIPLM_ERR_UNSUPPORTED (group_size > 64),
+ * ZIPLM_ERR_WORKSPACE, ZIPLM_ERR_CUDA.
+ */
+size_t ziplm_prune_workspace_bytes(int L, int d_row, int d_col, int group_size, int n_levels);
+
+ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row, int d_col,
+                                int group_size, float damp_frac, const int* levels, int n_levels,
+                                float* W_snap, float* loss, float* base_loss, int* order,
+                                float* saliency, int* layer_status, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZIPLM_H_ */

@@ -1,0 +1,82 @@
+// Shared host/device helpers for the ZipLM structured-OBS kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "ziplm.h"
+
+namespace ziplm {
+
+constexpr int kTile = 64;          // tile edge of the float64 factorisation kernels
+constexpr size_t kAlign = 256;     // alignment of every carve-out of a workspace
+
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+inline int round_up_int(int x, int a) { return (x + a - 1) / a * a; }
+
+// Bump allocator over a caller-provided workspace; with base == nullptr it only measures.
+struct Carver {
+    char* base;
+    size_t off;
+    explicit Carver(void* b) : base(static_cast<char*>(b)), off(0) {}
+    template <typename T>
+    T* take(size_t count) {
+        size_t start = off;
+        off = align_up(off + count * sizeof(T));
+        return base ? reinterpret_cast<T*>(base + start) : nullptr;
+    }
+};
+
+// Launch-error check used by the host planners: returns ZIPLM_ERR_CUDA from the caller.
+#define ZIPLM_CHECK_LAUNCH()                                   \
+    do {                                                       \
+        cudaError_t e__ = cudaGetLastError();                  \
+        if (e__ != cudaSuccess) return ZIPLM_ERR_CUDA;         \
+    } while (0)
+
+#define ZIPLM_CHECK_CUDA(expr)                                 \
+    do {                                                       \
+        cudaError_t e__ = (expr);                              \
+        if (e__ != cudaSuccess) return ZIPLM_ERR_CUDA;         \
+    } while (0)
+
+// A layer's status only ever moves from OK to the first error seen.
+__device__ inline void set_layer_status(int* layer_status, int l, int code) {
+    atomicCAS(layer_status + l, (int)ZIPLM_OK, code);
+}
+
+// ---- stages implemented in the other translation units (host-side planners) -----------------
+
+// Workspace of the float64 damped inverse for L layers of width d.
+size_t inverse_workspace_bytes(int L, int d);
+
+// (H + lambda I)^-1 in float64.  out64 (may be null) receives the full symmetric [L, d, d]
+// matrix; tri32/diag64 (may be null) receive the strictly lower triangle in fp32 with row pitch
+// `pitch32` and the diagonal in float64; lam_out (may be null) receives lambda per layer.
+ziplm_status run_damped_inverse(const float* H, int L, int d, float damp_frac, double* out64,
+                                float* tri32, int pitch32, double* diag64, double* lam_out,
+                                int* layer_status, void* ws, size_t ws_bytes, cudaStream_t st);
+
+size_t neuron_workspace_bytes(int L, int r, int d, int n_levels);
+ziplm_status run_prune_neurons(const float* W, const float* H, int L, int r, int d,
+                               float damp_frac, const int* levels, int n_levels, float* W_snap,
+                               float* loss, float* base_loss, int* order, float* saliency,
+                               int* layer_status, void* ws, size_t ws_bytes, cudaStream_t st);
+
+size_t block_workspace_bytes(int L, int r, int d, int g, int n_levels);
+ziplm_status run_prune_blocks(const float* W, const float* H, int L, int r, int d, int g,
+                              float damp_frac, const int* levels, int n_levels, float* W_snap,
+                              float* loss, float* base_loss, int* order, float* saliency,
+                              int* layer_status, void* ws, size_t ws_bytes, cudaStream_t st);
+
+// base_loss[l] = 1/2 tr(W[l] H[l] W[l]^T) = ||W X||_F^2; acc64 is an [L] float64 scratch.
+ziplm_status run_base_loss(const float* W, const float* H, int L, int r, int d, double* acc64,
+                           float* base_loss, cudaStream_t st);
+
+size_t hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt);
+ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, int L, int d, long long N,
+                         long long ldx, float alpha, float beta, void* ws, size_t ws_bytes,
+                         cudaStream_t st);
+
+}  // namespace ziplm
