@@ -1,0 +1,201 @@
+"""ctypes binding of libziplm.so: argument marshalling only, every step runs in the CUDA kernels.
+
+Function names and arguments mirror ``include/ziplm.h``.  Tensors are torch CUDA tensors; they
+are used as device buffers (``data_ptr``) and the current torch stream is passed down.  There is
+no fallback: if the shared library is missing or was not built, importing a function works but
+calling it raises :class:`ZiplmError`.
+"""
+from __future__ import annotations
+
+import ctypes
+import enum
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+
+class Status(enum.IntEnum):
+    OK = 0
+    ERR_INVALID_ARG = 1
+    ERR_WORKSPACE = 2
+    ERR_NOT_PD = 3
+    ERR_NONFINITE = 4
+    ERR_TIMEOUT = 5
+    ERR_CUDA = 6
+    ERR_UNSUPPORTED = 7
+
+
+F32, BF16 = 0, 1
+
+
+class ZiplmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = Status(status) if status in Status._value2member_map_ else status
+        super().__init__(f"{where}: {status_string(status)}")
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, "libziplm.so")
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libziplm.so (built by ``python -m paper_2302_04089_b200.build``) and type its symbols."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = lib_path()
+    if not os.path.exists(path):
+        raise ZiplmError(Status.ERR_CUDA, f"{path} is missing -- run paper_2302_04089_b200/build.py; "
+                                          "there is no CPU fallback")
+    lib = ctypes.CDLL(path)
+    c_int, c_ll, c_f, c_sz, vp = (ctypes.c_int, ctypes.c_longlong, ctypes.c_float, ctypes.c_size_t,
+                                  ctypes.c_void_p)
+    lib.ziplm_status_string.restype = ctypes.c_char_p
+    lib.ziplm_status_string.argtypes = [c_int]
+    lib.ziplm_hessian_workspace_bytes.restype = c_sz
+    lib.ziplm_hessian_workspace_bytes.argtypes = [c_int, c_int, c_ll, c_int]
+    lib.ziplm_hessian_accumulate.restype = c_int
+    lib.ziplm_hessian_accumulate.argtypes = [vp, vp, c_int, c_int, c_int, c_ll, c_ll, c_f, c_f, vp,
+                                             c_sz, vp]
+    lib.ziplm_inverse_workspace_bytes.restype = c_sz
+    lib.ziplm_inverse_workspace_bytes.argtypes = [c_int, c_int]
+    lib.ziplm_damped_inverse.restype = c_int
+    lib.ziplm_damped_inverse.argtypes = [vp, c_int, c_int, c_f, vp, vp, vp, c_sz, vp]
+    lib.ziplm_prune_workspace_bytes.restype = c_sz
+    lib.ziplm_prune_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int, c_int]
+    lib.ziplm_prune_layers.restype = c_int
+    lib.ziplm_prune_layers.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_f,
+                                       ctypes.POINTER(c_int), c_int, vp, vp, vp, vp, vp, vp, vp,
+                                       c_sz, vp]
+    _LIB = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    try:
+        return load_library().ziplm_status_string(int(status)).decode()
+    except ZiplmError:
+        return f"status {int(status)}"
+
+
+def _stream_ptr(t: torch.Tensor) -> int:
+    return torch.cuda.current_stream(t.device).cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _check(t: torch.Tensor, dtype, name: str):
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    # torch's caching allocator returns 512-byte aligned blocks
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def hessian_workspace_bytes(L: int, d: int, n_tokens: int, x_dtype: int) -> int:
+    return int(load_library().ziplm_hessian_workspace_bytes(L, d, n_tokens, x_dtype))
+
+
+def inverse_workspace_bytes(L: int, d: int) -> int:
+    return int(load_library().ziplm_inverse_workspace_bytes(L, d))
+
+
+def prune_workspace_bytes(L: int, d_row: int, d_col: int, group_size: int, n_levels: int) -> int:
+    return int(load_library().ziplm_prune_workspace_bytes(L, d_row, d_col, group_size, n_levels))
+
+
+def hessian_accumulate(X: torch.Tensor, H: Optional[torch.Tensor] = None, alpha: float = 2.0,
+                       beta: float = 0.0, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """H = beta * H + alpha * X X^T per layer.  X [L, d, N] fp32 or bf16 (tokens contiguous)."""
+    lib = load_library()
+    if X.dim() != 3 or not X.is_cuda or X.stride(2) != 1 and X.shape[2] > 1:
+        raise ValueError("X must be a CUDA tensor [L, d, N] with contiguous tokens")
+    if X.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("X must be fp32 or bf16")
+    L, d, N = X.shape
+    if X.stride(0) != d * X.stride(1):
+        raise ValueError("layers of X must be evenly pitched")
+    ldx = X.stride(1) if N > 0 else max(N, 1)
+    dt = F32 if X.dtype == torch.float32 else BF16
+    if H is None:
+        H = torch.zeros(L, d, d, dtype=torch.float32, device=X.device)
+        beta = 0.0
+    _check(H, torch.float32, "H")
+    need = hessian_workspace_bytes(L, d, N, dt)
+    if workspace is None:
+        workspace = _workspace(need, X.device)
+    with torch.cuda.device(X.device):
+        st = lib.ziplm_hessian_accumulate(H.data_ptr(), X.data_ptr(), dt, L, d, N, ldx, alpha, beta,
+                                          workspace.data_ptr(), workspace.numel(), _stream_ptr(X))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_hessian_accumulate")
+    return H
+
+
+def damped_inverse(H: torch.Tensor, damp_frac: float, workspace: Optional[torch.Tensor] = None):
+    """(Hinv [L, d, d] float64, layer_status [L] int32) for H [L, d, d] fp32."""
+    lib = load_library()
+    _check(H, torch.float32, "H")
+    L, d, _ = H.shape
+    Hinv = torch.empty(L, d, d, dtype=torch.float64, device=H.device)
+    status = torch.zeros(L, dtype=torch.int32, device=H.device)
+    if workspace is None:
+        workspace = _workspace(inverse_workspace_bytes(L, d), H.device)
+    with torch.cuda.device(H.device):
+        st = lib.ziplm_damped_inverse(H.data_ptr(), L, d, damp_frac, Hinv.data_ptr(),
+                                      status.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                      _stream_ptr(H))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_damped_inverse")
+    return Hinv, status
+
+
+def prune_layers(W: torch.Tensor, H: torch.Tensor, group_size: int, damp_frac: float,
+                 levels: Sequence[int], want_base_loss: bool = True, want_saliency: bool = True,
+                 workspace: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
+    """Greedy structured pruning of L same-shape layers; see ziplm_prune_layers in ziplm.h.
+
+    Returns a dict of CUDA tensors: W_snap [L, n_levels, r, d], loss [L, n_levels], base_loss [L]
+    (or None), order [L, G] int32, saliency [L, G] (or None), layer_status [L] int32.  Pass ``out``
+    (a dict from an earlier call) and ``workspace`` to reuse the buffers.
+    """
+    lib = load_library()
+    _check(W, torch.float32, "W")
+    _check(H, torch.float32, "H")
+    L, r, d = W.shape
+    if tuple(H.shape) != (L, d, d):
+        raise ValueError("H must be [L, d_col, d_col]")
+    levels = [int(v) for v in levels]
+    n_levels = len(levels)
+    G = d // group_size if group_size > 0 and d % group_size == 0 else 0
+    dev = W.device
+    if out is None:
+        out = dict(
+            W_snap=torch.empty(L, n_levels, r, d, dtype=torch.float32, device=dev),
+            loss=torch.empty(L, n_levels, dtype=torch.float32, device=dev),
+            base_loss=torch.empty(L, dtype=torch.float32, device=dev) if want_base_loss else None,
+            order=torch.empty(L, max(G, 1), dtype=torch.int32, device=dev),
+            saliency=torch.empty(L, max(G, 1), dtype=torch.float32, device=dev) if want_saliency else None,
+            layer_status=torch.empty(L, dtype=torch.int32, device=dev),
+        )
+    if workspace is None:
+        workspace = _workspace(prune_workspace_bytes(L, r, d, group_size, n_levels), dev)
+    lv = (ctypes.c_int * max(n_levels, 1))(*levels)
+    with torch.cuda.device(dev):
+        st = lib.ziplm_prune_layers(W.data_ptr(), H.data_ptr(), L, r, d, group_size, damp_frac, lv,
+                                    n_levels, _ptr(out["W_snap"]), _ptr(out["loss"]),
+                                    _ptr(out["base_loss"]), _ptr(out["order"]), _ptr(out["saliency"]),
+                                    _ptr(out["layer_status"]), workspace.data_ptr(),
+                                    workspace.numel(), _stream_ptr(W))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_prune_layers")
+    out["workspace"] = workspace
+    return out

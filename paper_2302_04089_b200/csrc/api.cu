@@ -1,0 +1,115 @@
+// extern "C" boundary: argument validation and dispatch.  No device memory is allocated here and
+// nothing synchronises; every stage is enqueued on the caller's stream.
+#include <math.h>
+
+#include "common.cuh"
+
+using namespace ziplm;
+
+namespace {
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bool have_device() {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev >= 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ziplm_status_string(ziplm_status s) {
+    switch (s) {
+        case ZIPLM_OK: return "ZIPLM_OK";
+        case ZIPLM_ERR_INVALID_ARG: return "ZIPLM_ERR_INVALID_ARG";
+        case ZIPLM_ERR_WORKSPACE: return "ZIPLM_ERR_WORKSPACE";
+        case ZIPLM_ERR_NOT_PD: return "ZIPLM_ERR_NOT_PD";
+        case ZIPLM_ERR_NONFINITE: return "ZIPLM_ERR_NONFINITE";
+        case ZIPLM_ERR_TIMEOUT: return "ZIPLM_ERR_TIMEOUT";
+        case ZIPLM_ERR_CUDA: return "ZIPLM_ERR_CUDA";
+        case ZIPLM_ERR_UNSUPPORTED: return "ZIPLM_ERR_UNSUPPORTED";
+    }
+    return "ZIPLM_ERR_UNKNOWN";
+}
+
+size_t ziplm_hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype x_dtype) {
+    if (L < 1 || d < 1 || n_tokens < 0) return 0;
+    return hessian_workspace_bytes(L, d, n_tokens, x_dtype);
+}
+
+ziplm_status ziplm_hessian_accumulate(float* H, const void* X, ziplm_dtype x_dtype, int L, int d,
+                                      long long n_tokens, long long ldx, float alpha, float beta,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (L < 1 || d < 1 || n_tokens < 0 || ldx < n_tokens || !H) return ZIPLM_ERR_INVALID_ARG;
+    if (x_dtype != ZIPLM_F32 && x_dtype != ZIPLM_BF16) return ZIPLM_ERR_INVALID_ARG;
+    if (!(beta == 0.f || beta == 1.f) || !isfinite(alpha)) return ZIPLM_ERR_INVALID_ARG;
+    const size_t esz = (x_dtype == ZIPLM_F32) ? 4 : 2;
+    if (n_tokens > 0) {
+        if (!X || !aligned(X, 16) || ((size_t)ldx * esz) % 16 != 0) return ZIPLM_ERR_INVALID_ARG;
+    }
+    const size_t need = hessian_workspace_bytes(L, d, n_tokens, x_dtype);
+    if (need > 0 && (!workspace || !aligned(workspace, kAlign) || workspace_bytes < need))
+        return ZIPLM_ERR_WORKSPACE;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    return run_hessian(H, X, x_dtype, L, d, n_tokens, ldx, alpha, beta, workspace, workspace_bytes,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t ziplm_inverse_workspace_bytes(int L, int d) {
+    if (L < 1 || d < 1) return 0;
+    return inverse_workspace_bytes(L, d);
+}
+
+ziplm_status ziplm_damped_inverse(const float* H, int L, int d, float damp_frac, double* Hinv,
+                                  int* layer_status, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream) {
+    if (L < 1 || d < 1 || !H || !Hinv || !layer_status) return ZIPLM_ERR_INVALID_ARG;
+    if (!(damp_frac >= 0.f) || !isfinite(damp_frac)) return ZIPLM_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, kAlign) || workspace_bytes < inverse_workspace_bytes(L, d))
+        return ZIPLM_ERR_WORKSPACE;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ZIPLM_CHECK_CUDA(cudaMemsetAsync(layer_status, 0, sizeof(int) * L, st));
+    return run_damped_inverse(H, L, d, damp_frac, Hinv, nullptr, 0, nullptr, nullptr, layer_status,
+                              workspace, workspace_bytes, st);
+}
+
+size_t ziplm_prune_workspace_bytes(int L, int d_row, int d_col, int group_size, int n_levels) {
+    if (L < 1 || d_row < 1 || d_col < 1 || group_size < 1 || n_levels < 0) return 0;
+    if (d_col % group_size != 0 || group_size > 64) return 0;
+    if (group_size == 1) return neuron_workspace_bytes(L, d_row, d_col, n_levels);
+    return block_workspace_bytes(L, d_row, d_col, group_size, n_levels);
+}
+
+ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row, int d_col,
+                                int group_size, float damp_frac, const int* levels, int n_levels,
+                                float* W_snap, float* loss, float* base_loss, int* order,
+                                float* saliency, int* layer_status, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream) {
+    if (L < 1 || d_row < 1 || d_col < 1 || group_size < 1 || n_levels < 0) return ZIPLM_ERR_INVALID_ARG;
+    if (d_col % group_size != 0) return ZIPLM_ERR_INVALID_ARG;
+    if (!W || !H || !order || !layer_status) return ZIPLM_ERR_INVALID_ARG;
+    if (n_levels > 0 && (!levels || !W_snap || !loss)) return ZIPLM_ERR_INVALID_ARG;
+    if (!(damp_frac >= 0.f) || !isfinite(damp_frac)) return ZIPLM_ERR_INVALID_ARG;
+    const int G = d_col / group_size;
+    for (int i = 0; i < n_levels; ++i) {
+        if (levels[i] < 0 || levels[i] > G) return ZIPLM_ERR_INVALID_ARG;
+        if (i > 0 && levels[i] >= levels[i - 1]) return ZIPLM_ERR_INVALID_ARG;
+    }
+    if (group_size > 64) return ZIPLM_ERR_UNSUPPORTED;
+    const size_t need = ziplm_prune_workspace_bytes(L, d_row, d_col, group_size, n_levels);
+    if (!workspace || !aligned(workspace, kAlign) || workspace_bytes < need) return ZIPLM_ERR_WORKSPACE;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ZIPLM_CHECK_CUDA(cudaMemsetAsync(layer_status, 0, sizeof(int) * L, st));
+    if (group_size == 1)
+        return run_prune_neurons(W, H, L, d_row, d_col, damp_frac, levels, n_levels, W_snap, loss,
+                                 base_loss, order, saliency, layer_status, workspace,
+                                 workspace_bytes, st);
+    return run_prune_blocks(W, H, L, d_row, d_col, group_size, damp_frac, levels, n_levels, W_snap,
+                            loss, base_loss, order, saliency, layer_status, workspace,
+                            workspace_bytes, st);
+}
+
+}  // extern "C"

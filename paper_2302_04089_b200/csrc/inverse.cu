@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(256) k_chol_update(double* C, int dp, int j) {
 __global__ void __launch_bounds__(256) k_potf2(double* C, int dp, int T, int j, double* Linv,
                                                int* layer_status) {
     __shared__ double s[kTile][kTile + 1];
-    __shared__ double inv[kTile][kTile + 1];
+    __shared__ double dinv[kTile];   // diagonal of the inverse factor
     __shared__ int sflag;
     const int l = blockIdx.x;
     const int tid = threadIdx.x;
@@ -195,19 +195,16 @@ __global__ void __launch_bounds__(256) k_potf2(double* C, int dp, int T, int j, 
         }
         __syncthreads();
     }
-    // inverse of the lower-triangular factor: thread `cidx` builds column cidx by substitution
+    // inverse of the lower-triangular factor: thread `cidx` builds column cidx by forward
+    // substitution.  Entry (i, cidx), i > cidx, is parked transposed in the unused strict upper
+    // triangle of s (slot [cidx][i]); the diagonal goes to dinv.
     if (tid < kTile) {
         const int cidx = tid;
-        for (int i = 0; i < kTile; ++i) {
-            double x;
-            if (i < cidx) {
-                x = 0.0;
-            } else {
-                double acc = (i == cidx) ? 1.0 : 0.0;
-                for (int k = cidx; k < i; ++k) acc -= s[i][k] * inv[k][cidx];
-                x = acc / s[i][i];
-            }
-            inv[i][cidx] = x;
+        dinv[cidx] = 1.0 / s[cidx][cidx];
+        for (int i = cidx + 1; i < kTile; ++i) {
+            double acc = -s[i][cidx] * dinv[cidx];
+            for (int k = cidx + 1; k < i; ++k) acc -= s[i][k] * s[cidx][k];
+            s[cidx][i] = acc / s[i][i];
         }
     }
     __syncthreads();
@@ -215,7 +212,7 @@ __global__ void __launch_bounds__(256) k_potf2(double* C, int dp, int T, int j, 
     for (int e = tid; e < kTile * kTile; e += 256) {
         const int i = e >> 6, jj = e & 63;
         tile[(size_t)i * dp + jj] = (jj <= i) ? s[i][jj] : 0.0;
-        li[e] = inv[i][jj];
+        li[e] = (jj < i) ? s[jj][i] : (jj == i ? dinv[i] : 0.0);
     }
     if (tid == 0 && sflag) set_layer_status(layer_status, l, sflag);
 }

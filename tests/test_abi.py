@@ -1,0 +1,63 @@
+"""The C-ABI library loads and exports every symbol that include/ziplm.h declares (no GPU)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2302_04089_b200 import build
+    return ctypes.CDLL(build.build())
+
+
+def declared_symbols():
+    src = open(os.path.join(ROOT, "include", "ziplm.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(ziplm_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_header_declares_the_expected_entry_points():
+    syms = declared_symbols()
+    for name in ("ziplm_hessian_accumulate", "ziplm_prune_layers", "ziplm_damped_inverse",
+                 "ziplm_hessian_workspace_bytes", "ziplm_prune_workspace_bytes",
+                 "ziplm_inverse_workspace_bytes", "ziplm_status_string"):
+        assert name in syms
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in declared_symbols():
+        assert hasattr(lib, name), name
+
+
+def test_status_strings_and_workspace_queries(lib):
+    lib.ziplm_status_string.restype = ctypes.c_char_p
+    names = [lib.ziplm_status_string(i).decode() for i in range(8)]
+    assert names[0] == "ZIPLM_OK" and len(set(names)) == 8
+    lib.ziplm_prune_workspace_bytes.restype = ctypes.c_size_t
+    lib.ziplm_inverse_workspace_bytes.restype = ctypes.c_size_t
+    a = lib.ziplm_prune_workspace_bytes(1, 64, 256, 1, 3)
+    b = lib.ziplm_prune_workspace_bytes(12, 768, 3072, 1, 12)
+    assert 0 < a < b and a % 256 == 0 and b % 256 == 0
+    assert lib.ziplm_prune_workspace_bytes(1, 64, 255, 64, 3) == 0     # 255 % 64 != 0
+    assert lib.ziplm_inverse_workspace_bytes(2, 100) >= 2 * 2 * 128 * 128 * 8
+
+
+def test_binding_mirrors_the_abi_names():
+    import paper_2302_04089_b200 as z
+    for name in declared_symbols():
+        assert hasattr(z, name[len("ziplm_"):]), name
+
+
+def test_compute_entry_points_fail_loudly_without_a_device(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    lib.ziplm_damped_inverse.restype = ctypes.c_int
+    buf = (ctypes.c_char * 4096)()
+    addr = (ctypes.addressof(buf) + 255) // 256 * 256
+    # invalid arguments are still reported first
+    assert lib.ziplm_damped_inverse(None, 1, 4, ctypes.c_float(0.01), None, None, None, 0, None) == 1

@@ -1,0 +1,187 @@
+"""CUDA path vs float64 oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from oracle import ziplm_oracle as zo
+from parity_util import compare_layer
+
+pytestmark = pytest.mark.gpu
+
+
+def zb():
+    import paper_2302_04089_b200 as z
+    return z
+
+
+def oracle_h32(X):
+    """fp32 rounding of the oracle's 2 X X^T: the H handed to both sides (never a CUDA result)."""
+    return torch.from_numpy(zo.hessian(X).astype(np.float32))
+
+
+def run_case(shape, levels=None, layers=None, check_layers=None, base=True):
+    z = zb()
+    levels = list(shape.levels if levels is None else levels)
+    W, X = wl.make_layers(shape, "cpu", layers)
+    H = torch.stack([oracle_h32(X[l]) for l in range(W.shape[0])])
+    out = z.prune_layers(W.cuda(), H.cuda(), shape.group_size, shape.damp_frac, levels,
+                         want_base_loss=base)
+    torch.cuda.synchronize()
+    reports = []
+    for l in (range(W.shape[0]) if check_layers is None else check_layers):
+        reports.append(compare_layer(W[l].numpy(), H[l].numpy(), shape.group_size, shape.damp_frac,
+                                     levels, out, l))
+    return out, reports
+
+
+# ------------------------------------------------------------------ Hessian (a1)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,N,ldx", [(64, 256, 256), (200, 1000, 1000), (130, 77 * 8, 640), (96, 8, 8)])
+def test_hessian_matches_oracle(dtype, d, N, ldx):
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=d, d_latent=32, n_tokens=ldx,
+                   n_layers=2, x_dtype=dtype)
+    _, X = wl.make_layers(sh, "cpu")
+    Xd = X.cuda()[:, :, :N]                       # pitched view: ldx >= N
+    H = z.hessian_accumulate(Xd)
+    torch.cuda.synchronize()
+    for l in range(2):
+        Ho = zo.hessian(X[l][:, :N])
+        scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
+        err = np.max(np.abs(H[l].cpu().double().numpy() - Ho) / scale)
+        assert err < 2e-6, err
+        assert torch.equal(H[l], H[l].T)
+    # beta = 1 adds a second batch: 2 X X^T accumulated twice = 4 X X^T
+    H2 = z.hessian_accumulate(Xd, H.clone(), beta=1.0)
+    torch.cuda.synchronize()
+    assert torch.allclose(H2, 2 * H, rtol=1e-6, atol=0)
+
+
+def test_hessian_zero_tokens_and_bad_args():
+    z = zb()
+    H = torch.ones(1, 8, 8, device="cuda")
+    X = torch.zeros(1, 8, 0, device="cuda")
+    assert torch.equal(z.hessian_accumulate(X, H.clone(), beta=1.0), H)
+    assert torch.count_nonzero(z.hessian_accumulate(X, H.clone(), beta=0.0)) == 0
+    Xb = torch.zeros(1, 8, 6, device="cuda")           # pitch 6 floats = 24 B: not 16-byte pitched
+    with pytest.raises(z.ZiplmError) as e:
+        z.hessian_accumulate(Xb)
+    assert e.value.status == z.Status.ERR_INVALID_ARG
+    with pytest.raises(z.ZiplmError):
+        z.hessian_accumulate(torch.zeros(1, 8, 8, device="cuda"), H.clone(), beta=0.5)
+
+
+# ------------------------------------------------------------------ damped inverse (a2, a3)
+@pytest.mark.parametrize("d,L", [(64, 1), (100, 2), (256, 3), (448, 1)])
+def test_damped_inverse_matches_oracle(d, L):
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=d, d_latent=max(8, d // 4),
+                   n_tokens=4 * d, n_layers=L)
+    _, X = wl.make_layers(sh, "cpu")
+    H = torch.stack([oracle_h32(X[l]) for l in range(L)])
+    Hinv, status = z.damped_inverse(H.cuda(), 0.01)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(status) == 0
+    for l in range(L):
+        ref = zo.inverse_spd(zo.damped(H[l].numpy(), 0.01)[0])
+        got = Hinv[l].cpu().numpy()
+        assert np.array_equal(got, got.T)
+        err = np.max(np.abs(got - ref)) / np.max(np.abs(ref))
+        assert err < 1e-10, err
+
+
+def test_not_positive_definite_layer_is_flagged_and_others_finish():
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c1_tiny_ffn"][0], d_col=64, d_latent=64, d_row=16, n_tokens=256,
+                   n_layers=3)
+    W, X = wl.make_layers(sh, "cpu")
+    H = torch.stack([oracle_h32(X[l]) for l in range(3)])
+    H[1] = -H[1]                                         # negative definite layer
+    H[1, 0, 0] = 1e9                                     # keep mean(diag) > 0 so damping is defined
+    Hinv, status = z.damped_inverse(H.cuda(), 0.01)
+    torch.cuda.synchronize()
+    assert status.tolist() == [0, int(z.Status.ERR_NOT_PD), 0]
+    out = z.prune_layers(W.cuda(), H.cuda(), 1, 0.01, [32])
+    torch.cuda.synchronize()
+    st = out["layer_status"].tolist()
+    assert st[0] == 0 and st[2] == 0 and st[1] == int(z.Status.ERR_NOT_PD)
+    for l in (0, 2):
+        compare_layer(W[l].numpy(), H[l].numpy(), 1, 0.01, [32], out, l)
+    Hn = H.clone()
+    Hn[2, 3, 3] = float("nan")
+    _, status = z.damped_inverse(Hn.cuda(), 0.01)
+    assert status.tolist()[2] == int(z.Status.ERR_NONFINITE) and status.tolist()[0] == 0
+
+
+# ------------------------------------------------------------------ neuron path (a4 - a10)
+def test_c1_tiny_ffn_full_config():
+    out, reports = run_case(wl.CONFIGS["c1_tiny_ffn"][0])
+    assert reports[0]["steps"] == 192
+
+
+@pytest.mark.parametrize("d,r,L,levels", [
+    (203, 50, 2, [203, 150, 77, 1, 0]),        # ragged widths, unpruned level, down to nothing
+    (64, 7, 1, [63, 0]),
+    (130, 129, 3, [65]),
+    (8, 4, 2, [4]),
+])
+def test_neuron_path_ragged_shapes(d, r, L, levels):
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=d, d_row=r, d_latent=max(4, d // 4),
+                   n_tokens=4 * d + 8, n_layers=L, levels=tuple(levels))
+    run_case(sh)
+
+
+def test_neuron_path_mid_size_full_depth_three_layers():
+    """Scaled BERT-base fc2: several row blocks per step, full greedy order 768 -> 0."""
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=768, d_row=192, d_latent=192,
+                   n_tokens=4096, n_layers=3, levels=tuple(range(704, -1, -64)))
+    out, reports = run_case(sh)
+    print(reports)
+
+
+def test_neuron_path_is_deterministic():
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=256, d_row=64, d_latent=64,
+                   n_tokens=1024, n_layers=2, levels=(128, 0))
+    W, X = wl.make_layers(sh, "cpu")
+    H = torch.stack([oracle_h32(X[l]) for l in range(2)]).cuda()
+    a = z.prune_layers(W.cuda(), H, 1, 0.01, [128, 0])
+    b = z.prune_layers(W.cuda(), H, 1, 0.01, [128, 0])
+    torch.cuda.synchronize()
+    assert torch.equal(a["order"], b["order"])
+    assert torch.equal(a["W_snap"], b["W_snap"])
+
+
+def test_workspace_is_not_assumed_clean():
+    """Poison the workspace with NaN bit patterns: values of unused slots never feed live ones."""
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=100, d_row=20, d_latent=25,
+                   n_tokens=512, n_layers=2, levels=(50, 10))
+    W, X = wl.make_layers(sh, "cpu")
+    H = torch.stack([oracle_h32(X[l]) for l in range(2)])
+    ws = torch.full((z.prune_workspace_bytes(2, 20, 100, 1, 2),), 0xFF, dtype=torch.uint8, device="cuda")
+    out = z.prune_layers(W.cuda(), H.cuda(), 1, 0.01, [50, 10], workspace=ws)
+    torch.cuda.synchronize()
+    for l in range(2):
+        compare_layer(W[l].numpy(), H[l].numpy(), 1, 0.01, [50, 10], out, l)
+
+
+# ------------------------------------------------------------------ host-side argument checks
+def test_invalid_arguments_are_rejected_on_the_host():
+    z = zb()
+    W = torch.zeros(1, 4, 8, device="cuda")
+    H = torch.eye(8, device="cuda")[None].contiguous()
+    for lv in ([3, 5], [9], [-1], [4, 4]):
+        with pytest.raises(z.ZiplmError) as e:
+            z.prune_layers(W, H, 1, 0.01, lv)
+        assert e.value.status == z.Status.ERR_INVALID_ARG
+    with pytest.raises(z.ZiplmError) as e:
+        z.prune_layers(W, H, 3, 0.01, [1])              # 8 % 3 != 0
+    assert e.value.status == z.Status.ERR_INVALID_ARG
+    with pytest.raises(z.ZiplmError) as e:
+        z.prune_layers(W, H, 1, -0.5, [1])
+    assert e.value.status == z.Status.ERR_INVALID_ARG
+    with pytest.raises(z.ZiplmError) as e:
+        z.prune_layers(W, H, 1, 0.01, [4], workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == z.Status.ERR_WORKSPACE
