@@ -179,7 +179,7 @@ __global__ void __launch_bounds__(256) k_potf2(double* C, int dp, int T, int j, 
         if (tid == 0) {
             double p = s[c][c];
             if (!(p > 0.0) || !isfinite(p)) {   // not positive definite (or NaN): flag, keep going
-                sflag = isfinite(p) ? ZIPLM_ERR_NOT_PD : ZIPLM_ERR_NONFINITE;
+                if (!sflag) sflag = isfinite(p) ? ZIPLM_ERR_NOT_PD : ZIPLM_ERR_NONFINITE;
                 p = 1.0;
             }
             s[c][c] = sqrt(p);

@@ -84,11 +84,15 @@ def test_damped_inverse_matches_oracle(d, L):
     torch.cuda.synchronize()
     assert torch.count_nonzero(status) == 0
     for l in range(L):
-        ref = zo.inverse_spd(zo.damped(H[l].numpy(), 0.01)[0])
+        H_lam = zo.damped(H[l].numpy(), float(np.float32(0.01)))[0]
+        ref = zo.inverse_spd(H_lam)
         got = Hinv[l].cpu().numpy()
         assert np.array_equal(got, got.T)
+        # float64 on both sides: forward error of an inverse is bounded by ~ cond * unit roundoff
+        tol = 50 * np.linalg.cond(H_lam) * 2.2e-16
         err = np.max(np.abs(got - ref)) / np.max(np.abs(ref))
-        assert err < 1e-10, err
+        assert err < tol, (err, tol)
+        assert np.max(np.abs(got @ H_lam - np.eye(d))) < tol * 10
 
 
 def test_not_positive_definite_layer_is_flagged_and_others_finish():
@@ -97,8 +101,7 @@ def test_not_positive_definite_layer_is_flagged_and_others_finish():
                    n_layers=3)
     W, X = wl.make_layers(sh, "cpu")
     H = torch.stack([oracle_h32(X[l]) for l in range(3)])
-    H[1] = -H[1]                                         # negative definite layer
-    H[1, 0, 0] = 1e9                                     # keep mean(diag) > 0 so damping is defined
+    H[1, 0, 1] = H[1, 1, 0] = 100.0 * H[1, 0, 0]         # indefinite even after 1 % damping
     Hinv, status = z.damped_inverse(H.cuda(), 0.01)
     torch.cuda.synchronize()
     assert status.tolist() == [0, int(z.Status.ERR_NOT_PD), 0]
