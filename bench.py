@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Throughput of the whole ZipLM layer-wise pruning path on synthetic BERT-base fc2 layers.
+
+One step = one pass of the whole path over one batch of 12 same-shape layers (W 768 x 3072,
+X 3072 x 16384 fp32): Hessian accumulation, damping + float64 Cholesky inverse, the full greedy
+loop 3072 -> 0 neurons, and a snapshot + loss at every 256 neurons.  The metric is pruned
+structures per second (12 * 3072 structures per step and per GPU).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  ``--impl reference`` times the float64 CPU oracle on a bounded
+sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import workloads as wl
+
+WORKLOAD = "c3_bert_base_fc2"
+METRIC = "pruned_structures_per_sec"
+UNIT = "structures/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle leg
+# ------------------------------------------------------------------------------------------
+def oracle_sample(shape, n_loop_steps=24):
+    """Time the float64 oracle, as it stands, on one layer of the workload: full Hessian, full
+    damped inverse, the first ``n_loop_steps`` greedy steps (every oracle step costs the same:
+    it updates the full d x d matrix).  Returns structures/s extrapolated to the full greedy
+    order of that layer, and the parts."""
+    from oracle import ziplm_oracle as zo
+    W = wl.make_weight(shape, 0)
+    X = wl.make_activations(shape, 0, "cpu")
+    t0 = time.perf_counter()
+    H = zo.hessian(X)
+    t1 = time.perf_counter()
+    H32 = H.astype(np.float32)
+    t2 = time.perf_counter()
+    res = zo.prune(W.numpy(), H32, shape.group_size, float(np.float32(shape.damp_frac)),
+                   [shape.n_groups - n_loop_steps], max_steps=n_loop_steps)
+    t3 = time.perf_counter()
+    # prune() = damping + inverse + n_loop_steps steps (+ one snapshot/loss); split by a second
+    # timing of the inverse alone
+    t4 = time.perf_counter()
+    zo.inverse_spd(zo.damped(H32, shape.damp_frac)[0])
+    t5 = time.perf_counter()
+    t_h, t_inv = t1 - t0, t5 - t4
+    t_step = max((t3 - t2) - t_inv, 1e-9) / n_loop_steps
+    G = shape.n_groups
+    t_layer = t_h + t_inv + t_step * G
+    return dict(value=G / t_layer, hessian_s=t_h, inverse_s=t_inv, step_s=t_step,
+                layer_s_extrapolated=t_layer, steps_timed=n_loop_steps,
+                order_head=[int(v) for v in res["order"][:4]])
+
+
+def cpu_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, shape):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(args.warmup):
+        oracle_sample(shape, n_loop_steps=2)
+    vals, t0 = [], time.perf_counter()
+    for _ in range(args.steps):
+        vals.append(oracle_sample(shape, n_loop_steps=args.oracle_steps))
+    dt = time.perf_counter() - t0
+    v = float(np.mean([s["value"] for s in vals]))
+    sample = (f"1 of {shape.n_layers} layers: full float64 Hessian + damped inverse + first "
+              f"{args.oracle_steps} of {shape.n_groups} greedy steps, extrapolated to the full order")
+    line = dict(impl="reference", metric=METRIC, value=v, unit=UNIT, n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * dt / max(args.steps, 1),
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64",
+                data="synthetic", config=dict(workload=WORKLOAD, layers=shape.n_layers,
+                                              d_row=shape.d_row, d_col=shape.d_col,
+                                              n_tokens=shape.n_tokens, group_size=shape.group_size),
+                cpu_baseline=dict(value=v, unit=UNIT, cores=cpu_cores(), kind="oracle", sample=sample),
+                e2e=dict(value=v, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); smax.append(float(parts[2])); power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        os.unlink(self.f.name)
+        # samples under load: the upper half by power draw
+        if sm:
+            order = np.argsort(power)
+            load = [sm[i] for i in order[len(order) // 2:]]
+            med = float(np.median(load))
+        else:
+            med = None
+        return dict(sm_mhz=med, sm_max_mhz=(max(smax) if smax else None), reasons=sorted(reasons),
+                    samples=len(sm), power_w_max=(max(power) if power else None))
+
+
+# ------------------------------------------------------------------------------------------
+# CUDA leg
+# ------------------------------------------------------------------------------------------
+def update_bytes(L, r, G):
+    """Algorithmic bytes of the fused H^-1 / W update over the whole greedy loop: per launch
+    with n live structures, L * (8 r n + 4 n^2) (read + write of the live W, read + write of one
+    triangle of H^-1).  The launch at n = 1 does not exist (nothing is left to update)."""
+    n = np.arange(2, G + 1, dtype=np.float64)
+    return float(L * np.sum(8.0 * r * n + 4.0 * n * n)), int(len(n))
+
+
+def run_ours(args, shape):
+    import paper_2302_04089_b200 as z
+    from paper_2302_04089_b200 import build as zbuild
+    zbuild.build()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+
+    L, r, d, N, g = shape.n_layers, shape.d_row, shape.d_col, shape.n_tokens, shape.group_size
+    G = shape.n_groups
+    levels = list(shape.levels)
+    # every rank prunes its own 12 layers (independent problems: no collective on the data path)
+    rs = wl.scaled(shape, seed_base=shape.seed_base + 100 * rank)
+    W, X = wl.make_layers(rs, dev)
+    torch.cuda.synchronize()
+    H = torch.empty(L, d, d, dtype=torch.float32, device=dev)
+    h_ws = torch.empty(max(z.hessian_workspace_bytes(L, d, N, 0), 256), dtype=torch.uint8, device=dev)
+    p_ws = torch.empty(z.prune_workspace_bytes(L, r, d, g, len(levels)), dtype=torch.uint8, device=dev)
+    out = None
+
+    def step():
+        nonlocal out
+        z.hessian_accumulate(X, H, alpha=2.0, beta=0.0, workspace=h_ws)
+        out = z.prune_layers(W, H, g, shape.damp_frac, levels, workspace=p_ws, out=out)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    assert int(torch.count_nonzero(out["layer_status"])) == 0, out["layer_status"].tolist()
+
+    # ---- device-resident timing
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = z.launch_count()
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1) / args.steps
+    launches = (z.launch_count() - launches0) // max(args.steps, 1)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the same calls with host buffers
+    Wh = W.cpu().pin_memory()
+    Xh = X.cpu().pin_memory()
+    host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory()
+                for k, v in out.items() if k in ("W_snap", "loss", "base_loss", "order", "layer_status")}
+    h2d = Wh.numel() * 4 + Xh.numel() * Xh.element_size()
+    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+
+    def e2e_step():
+        W.copy_(Wh, non_blocking=True)
+        X.copy_(Xh, non_blocking=True)
+        step()
+        for k, v in host_out.items():
+            v.copy_(out[k], non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 3))
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+
+    # ---- one more step with per-phase event timing (roofline of the update kernel)
+    z.profile_begin()
+    step()
+    torch.cuda.synchronize()
+    phases = z.profile_end()
+
+    if dist is not None:
+        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    structures = world * L * G
+    value = structures / (ms * 1e-3)
+    e2e_value = structures / (ms_e2e * 1e-3)
+
+    if rank == 0:
+        peak, peak_src = load_peaks()
+        upd_ms, upd_n = phases["update"]
+        alg_bytes, n_launch = update_bytes(L, r, G)
+        achieved = alg_bytes / (upd_ms * 1e-3) / 1e9 if upd_ms > 0 else 0.0
+        line = dict(
+            metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
+            warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
+            vs_baseline=None, dtype="f32", data="synthetic",
+            config=dict(workload=WORKLOAD, layers=L, d_row=r, d_col=d, n_tokens=N, group_size=g,
+                        levels=len(levels), damp_frac=shape.damp_frac,
+                        l2_policy="inputs_exceed_l2 (X 2.4 GB, H^-1 workspace 0.45 GB per step)",
+                        parallelism=f"layer-sharded x{world}, no collective"),
+            layers_per_sec=world * L / (ms * 1e-3),
+            phases_ms={k: round(v[0], 3) for k, v in phases.items() if v[1] > 0},
+            e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                     ms_per_step=ms_e2e),
+            gpu_launches=int(launches),
+            clocks=clocks,
+            roofline=dict(kernel="k_neuron_update", bound="hbm", achieved=achieved, peak=peak,
+                          unit="GB/s", frac=achieved / peak, traffic=None, peak_source=peak_src,
+                          launches=upd_n, avg_launch_us=1e3 * upd_ms / max(upd_n, 1),
+                          algorithmic_bytes_per_step=alg_bytes),
+        )
+        if world == 1 and not args.no_cpu_baseline:
+            s = oracle_sample(shape, n_loop_steps=args.oracle_steps)
+            line["cpu_baseline"] = dict(
+                value=s["value"], unit=UNIT, cores=cpu_cores(), kind="oracle",
+                sample=(f"1 of {L} layers: full float64 Hessian ({s['hessian_s']:.1f} s) + damped "
+                        f"inverse ({s['inverse_s']:.1f} s) + first {s['steps_timed']} of {G} greedy "
+                        f"steps ({s['step_s'] * 1e3:.0f} ms each), extrapolated to the full order"))
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--oracle-steps", type=int, default=24)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    shape = wl.CONFIGS[WORKLOAD][0]
+    if args.impl == "reference":
+        run_reference(args, shape)
+    else:
+        if args.warmup < 3:
+            args.warmup = 3          # timing rule: at least three warm-up steps
+        run_ours(args, shape)
+
+
+if __name__ == "__main__":
+    main()

@@ -6,7 +6,7 @@
  *   - "dev" pointers are CUDA device pointers of the current device, "host" pointers are
  *     ordinary host memory.  All matrices are dense row-major.
  *   - The caller owns every buffer.  The library allocates no device memory, creates no stream
- *     and keeps no state between calls.
+ *     and keeps no state between calls (the optional diagnostics at the end of this file aside).
  *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = the default
  *     stream) and the call returns without synchronising.  Buffers must stay alive until the
  *     stream has drained.
@@ -140,6 +140,25 @@ ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row
                                 float* W_snap, float* loss, float* base_loss, int* order,
                                 float* saliency, int* layer_status, void* workspace,
                                 size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Diagnostics (no counterpart in the paper): a launch counter and optional per-phase timing.
+ *
+ * ziplm_launch_count       kernels launched by this library since it was loaded.
+ * ziplm_profile_begin      from now on every phase of every call is bracketed by a pair of CUDA
+ *                          events on the caller's stream (process-wide switch, not re-entrant;
+ *                          costs a few microseconds per phase, so timed runs leave it off).
+ * ziplm_profile_end        switches timing off, waits for the recorded events and returns, per
+ *                          phase, the summed milliseconds (host [n_phases] double, may be NULL)
+ *                          and the number of bracketed spans (host [n_phases], may be NULL).
+ * ziplm_profile_phase_count / ziplm_profile_phase_name   enumerate the phases ("hessian",
+ *                          "inverse", "init", "prep", "update", "snapshot", ...).
+ */
+long long ziplm_launch_count(void);
+ziplm_status ziplm_profile_begin(void);
+ziplm_status ziplm_profile_end(double* phase_ms, long long* phase_spans, int n_phases);
+int ziplm_profile_phase_count(void);
+const char* ziplm_profile_phase_name(int phase);
 
 #ifdef __cplusplus
 }

@@ -71,6 +71,16 @@ def load_library() -> ctypes.CDLL:
     lib.ziplm_prune_layers.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_f,
                                        ctypes.POINTER(c_int), c_int, vp, vp, vp, vp, vp, vp, vp,
                                        c_sz, vp]
+    lib.ziplm_launch_count.restype = ctypes.c_longlong
+    lib.ziplm_launch_count.argtypes = []
+    lib.ziplm_profile_begin.restype = c_int
+    lib.ziplm_profile_begin.argtypes = []
+    lib.ziplm_profile_end.restype = c_int
+    lib.ziplm_profile_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(c_ll), c_int]
+    lib.ziplm_profile_phase_count.restype = c_int
+    lib.ziplm_profile_phase_count.argtypes = []
+    lib.ziplm_profile_phase_name.restype = ctypes.c_char_p
+    lib.ziplm_profile_phase_name.argtypes = [c_int]
     _LIB = lib
     return lib
 
@@ -199,3 +209,35 @@ def prune_layers(W: torch.Tensor, H: torch.Tensor, group_size: int, damp_frac: f
         raise ZiplmError(st, "ziplm_prune_layers")
     out["workspace"] = workspace
     return out
+
+
+def launch_count() -> int:
+    """Kernels launched by the library since it was loaded."""
+    return int(load_library().ziplm_launch_count())
+
+
+def profile_begin() -> None:
+    """Switch on per-phase CUDA-event timing for the calls that follow."""
+    st = load_library().ziplm_profile_begin()
+    if st != 0:
+        raise ZiplmError(st, "ziplm_profile_begin")
+
+
+def profile_end() -> dict:
+    """Switch timing off and return {phase name: (milliseconds, spans)} (synchronises)."""
+    lib = load_library()
+    n = lib.ziplm_profile_phase_count()
+    ms = (ctypes.c_double * n)()
+    cnt = (ctypes.c_longlong * n)()
+    st = lib.ziplm_profile_end(ms, cnt, n)
+    if st != 0:
+        raise ZiplmError(st, "ziplm_profile_end")
+    return {lib.ziplm_profile_phase_name(i).decode(): (ms[i], int(cnt[i])) for i in range(n)}
+
+
+def profile_phase_count() -> int:
+    return int(load_library().ziplm_profile_phase_count())
+
+
+def profile_phase_name(i: int) -> str:
+    return load_library().ziplm_profile_phase_name(i).decode()

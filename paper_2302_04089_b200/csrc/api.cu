@@ -52,6 +52,7 @@ ziplm_status ziplm_hessian_accumulate(float* H, const void* X, ziplm_dtype x_dty
     if (need > 0 && (!workspace || !aligned(workspace, kAlign) || workspace_bytes < need))
         return ZIPLM_ERR_WORKSPACE;
     if (!have_device()) return ZIPLM_ERR_CUDA;
+    PhaseScope ps(PH_HESSIAN, static_cast<cudaStream_t>(cuda_stream));
     return run_hessian(H, X, x_dtype, L, d, n_tokens, ldx, alpha, beta, workspace, workspace_bytes,
                        static_cast<cudaStream_t>(cuda_stream));
 }
@@ -71,6 +72,7 @@ ziplm_status ziplm_damped_inverse(const float* H, int L, int d, float damp_frac,
     if (!have_device()) return ZIPLM_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     ZIPLM_CHECK_CUDA(cudaMemsetAsync(layer_status, 0, sizeof(int) * L, st));
+    PhaseScope ps(PH_INVERSE, st);
     return run_damped_inverse(H, L, d, damp_frac, Hinv, nullptr, 0, nullptr, nullptr, layer_status,
                               workspace, workspace_bytes, st);
 }

@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <stddef.h>
+#include <atomic>
 #include <stdint.h>
 
 #include "ziplm.h"
@@ -28,9 +29,26 @@ struct Carver {
     }
 };
 
-// Launch-error check used by the host planners: returns ZIPLM_ERR_CUDA from the caller.
+// Number of kernels launched by this library since it was loaded (diagnostics).
+extern std::atomic<long long> g_launches;
+
+// Phases reported by the optional event timing (ziplm_profile_begin / ziplm_profile_end).
+enum Phase { PH_HESSIAN = 0, PH_INVERSE, PH_INIT, PH_PREP, PH_UPDATE, PH_SNAPSHOT, PH_BLOCK_SCORE,
+             PH_BLOCK_UPDATE, PH_COUNT };
+
+// Brackets the launches issued during its lifetime with a pair of events when timing is on.
+struct PhaseScope {
+    PhaseScope(int phase, cudaStream_t st);
+    ~PhaseScope();
+    cudaStream_t st_;
+    int idx_;
+};
+
+// Placed after every kernel launch: counts it and returns ZIPLM_ERR_CUDA from the caller if the
+// launch failed.
 #define ZIPLM_CHECK_LAUNCH()                                   \
     do {                                                       \
+        ++::ziplm::g_launches;                                 \
         cudaError_t e__ = cudaGetLastError();                  \
         if (e__ != cudaSuccess) return ZIPLM_ERR_CUDA;         \
     } while (0)

@@ -1,0 +1,87 @@
+// Diagnostics: launch counter and optional per-phase CUDA-event timing.  Off by default; when
+// switched on, every phase of the following calls is bracketed by a pair of events on the
+// caller's stream, which costs a little time between kernels but no device memory.
+#include <atomic>
+#include <mutex>
+#include <vector>
+
+#include "common.cuh"
+
+namespace ziplm {
+
+std::atomic<long long> g_launches{0};
+
+namespace {
+struct Span { int phase; cudaEvent_t a, b; };
+std::mutex g_mu;
+bool g_on = false;
+std::vector<Span> g_spans;
+const char* kPhaseNames[PH_COUNT] = {"hessian", "inverse", "init", "prep", "update", "snapshot",
+                                     "block_score", "block_update"};
+}  // namespace
+
+PhaseScope::PhaseScope(int phase, cudaStream_t st) : st_(st), idx_(-1) {
+    if (!g_on) return;
+    std::lock_guard<std::mutex> lk(g_mu);
+    Span s;
+    s.phase = phase;
+    if (cudaEventCreate(&s.a) != cudaSuccess) return;
+    if (cudaEventCreate(&s.b) != cudaSuccess) { cudaEventDestroy(s.a); return; }
+    cudaEventRecord(s.a, st);
+    g_spans.push_back(s);
+    idx_ = (int)g_spans.size() - 1;
+}
+
+PhaseScope::~PhaseScope() {
+    if (idx_ < 0) return;
+    std::lock_guard<std::mutex> lk(g_mu);
+    cudaEventRecord(g_spans[idx_].b, st_);
+}
+
+}  // namespace ziplm
+
+using namespace ziplm;
+
+extern "C" {
+
+long long ziplm_launch_count(void) { return g_launches.load(); }
+
+int ziplm_profile_phase_count(void) { return PH_COUNT; }
+
+const char* ziplm_profile_phase_name(int phase) {
+    return (phase >= 0 && phase < PH_COUNT) ? kPhaseNames[phase] : "?";
+}
+
+ziplm_status ziplm_profile_begin(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    for (auto& s : g_spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
+    g_spans.clear();
+    g_on = true;
+    return ZIPLM_OK;
+}
+
+ziplm_status ziplm_profile_end(double* phase_ms, long long* phase_spans, int n_phases) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_on = false;
+    for (int i = 0; i < n_phases; ++i) {
+        if (phase_ms) phase_ms[i] = 0.0;
+        if (phase_spans) phase_spans[i] = 0;
+    }
+    ziplm_status rc = ZIPLM_OK;
+    for (auto& s : g_spans) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(s.b) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, s.a, s.b) != cudaSuccess) {
+            rc = ZIPLM_ERR_CUDA;
+        } else if (s.phase < n_phases) {
+            if (phase_ms) phase_ms[s.phase] += (double)ms;
+            if (phase_spans) phase_spans[s.phase] += 1;
+        }
+        cudaEventDestroy(s.a);
+        cudaEventDestroy(s.b);
+    }
+    g_spans.clear();
+    return rc;
+}
+
+}  // extern "C"

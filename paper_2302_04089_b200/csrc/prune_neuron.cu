@@ -387,20 +387,29 @@ ziplm_status run_prune_neurons(const float* W, const float* H, int L, int r, int
     NeuronWs w = carve_neuron(ws, L, r, d);
     const int G = d;
 
-    ziplm_status s = run_damped_inverse(H, L, d, damp_frac, nullptr, w.A, w.pitch, w.diag, w.lam,
-                                        layer_status, w.inv_ws, w.inv_bytes, st);
-    if (s != ZIPLM_OK) return s;
-    ZIPLM_CHECK_CUDA(cudaMemsetAsync(order, 0xFF, sizeof(int) * (size_t)L * G, st));
-    if (saliency) ZIPLM_CHECK_CUDA(cudaMemsetAsync(saliency, 0, sizeof(float) * (size_t)L * G, st));
-    k_neuron_init<<<dim3((d + 31) / 32, L), 256, 0, st>>>(W, r, d, w.rp, w.Wt, w.diag, w.rho, w.idx,
-                                                         w.state);
-    ZIPLM_CHECK_LAUNCH();
-    if (base_loss) {
-        s = run_base_loss(W, H, L, r, d, w.base_acc, base_loss, st);
-        if (s != ZIPLM_OK) return s;
+    ziplm_status s;
+    {
+        PhaseScope ps(PH_INVERSE, st);
+        s = run_damped_inverse(H, L, d, damp_frac, nullptr, w.A, w.pitch, w.diag, w.lam, layer_status,
+                               w.inv_ws, w.inv_bytes, st);
     }
+    if (s != ZIPLM_OK) return s;
+    auto init = [&]() -> ziplm_status {
+        PhaseScope ps(PH_INIT, st);
+        ZIPLM_CHECK_CUDA(cudaMemsetAsync(order, 0xFF, sizeof(int) * (size_t)L * G, st));
+        if (saliency)
+            ZIPLM_CHECK_CUDA(cudaMemsetAsync(saliency, 0, sizeof(float) * (size_t)L * G, st));
+        k_neuron_init<<<dim3((d + 31) / 32, L), 256, 0, st>>>(W, r, d, w.rp, w.Wt, w.diag, w.rho,
+                                                             w.idx, w.state);
+        ZIPLM_CHECK_LAUNCH();
+        if (base_loss) return run_base_loss(W, H, L, r, d, w.base_acc, base_loss, st);
+        return ZIPLM_OK;
+    };
+    s = init();
+    if (s != ZIPLM_OK) return s;
 
     auto snapshot = [&](int n, int slot) -> ziplm_status {
+        PhaseScope ps(PH_SNAPSHOT, st);
         k_neuron_pos_of<<<L, 256, 0, st>>>(n, d, w.idx, w.pos_of);
         ZIPLM_CHECK_LAUNCH();
         k_neuron_snapshot<<<dim3((d + 31) / 32, (r + 31) / 32, L), 256, 0, st>>>(
@@ -418,10 +427,15 @@ ziplm_status run_prune_neurons(const float* W, const float* H, int L, int r, int
     }
     const int n_min = n_levels > 0 ? levels[n_levels - 1] : G;
     for (int t = 0; n > n_min; ++t) {
-        k_neuron_prep<<<L, 512, 0, st>>>(n, t, d, G, w.pitch, r, w.rp, w.A, w.Wt, w.diag, w.rho, w.idx,
-                                         w.ubuf, w.cbuf, w.state, order, saliency, layer_status);
-        ZIPLM_CHECK_LAUNCH();
+        {
+            PhaseScope ps(PH_PREP, st);
+            k_neuron_prep<<<L, 512, 0, st>>>(n, t, d, G, w.pitch, r, w.rp, w.A, w.Wt, w.diag, w.rho,
+                                             w.idx, w.ubuf, w.cbuf, w.state, order, saliency,
+                                             layer_status);
+            ZIPLM_CHECK_LAUNCH();
+        }
         if (n > 1) {
+            PhaseScope ps(PH_UPDATE, st);
             k_neuron_update<<<dim3((n + 7) / 8, L), 256, 0, st>>>(n, d, w.pitch, w.rp, w.A, w.Wt,
                                                                  w.diag, w.rho, w.ubuf, w.cbuf, w.state);
             ZIPLM_CHECK_LAUNCH();
