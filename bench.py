@@ -167,11 +167,11 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 # CUDA leg
 # ------------------------------------------------------------------------------------------
-def update_bytes(L, r, G):
+def update_bytes(L, r, G, n_removed):
     """Algorithmic bytes of the fused H^-1 / W update over the whole greedy loop: per launch
     with n live structures, L * (8 r n + 4 n^2) (read + write of the live W, read + write of one
     triangle of H^-1).  The launch at n = 1 does not exist (nothing is left to update)."""
-    n = np.arange(2, G + 1, dtype=np.float64)
+    n = np.arange(max(2, G - n_removed + 1), G + 1, dtype=np.float64)
     return float(L * np.sum(8.0 * r * n + 4.0 * n * n)), int(len(n))
 
 
@@ -251,15 +251,17 @@ def run_ours(args, shape):
         for k, v in host_out.items():
             v.copy_(out[k], non_blocking=True)
 
-    e2e_steps = max(1, min(args.steps, 3))
-    e2e_step()
-    barrier()
-    e0.record()
-    for _ in range(e2e_steps):
+    e2e_steps = 0 if args.skip_e2e else max(1, min(args.steps, 3))
+    ms_e2e = float("nan")
+    if e2e_steps:
         e2e_step()
-    e1.record()
-    barrier()
-    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        ms_e2e = e0.elapsed_time(e1) / e2e_steps
 
     # ---- one more step with per-phase event timing (roofline of the update kernel)
     z.profile_begin()
@@ -271,20 +273,22 @@ def run_ours(args, shape):
         t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms, ms_e2e = float(t[0]), float(t[1])
-    structures = world * L * G
+    n_removed = G - min(levels)
+    structures = world * L * n_removed
     value = structures / (ms * 1e-3)
     e2e_value = structures / (ms_e2e * 1e-3)
 
     if rank == 0:
         peak, peak_src = load_peaks()
         upd_ms, upd_n = phases["update"]
-        alg_bytes, n_launch = update_bytes(L, r, G)
+        alg_bytes, n_launch = update_bytes(L, r, G, n_removed)
         achieved = alg_bytes / (upd_ms * 1e-3) / 1e9 if upd_ms > 0 else 0.0
         line = dict(
             metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
             warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
             vs_baseline=None, dtype="f32", data="synthetic",
-            config=dict(workload=WORKLOAD, layers=L, d_row=r, d_col=d, n_tokens=N, group_size=g,
+            config=dict(workload=WORKLOAD if (args.layers == 0 and args.max_removed == 0)
+                        else WORKLOAD + " (reduced: profiling aid)", layers=L, d_row=r, d_col=d, n_tokens=N, group_size=g,
                         levels=len(levels), damp_frac=shape.damp_frac,
                         l2_policy="inputs_exceed_l2 (X 2.4 GB, H^-1 workspace 0.45 GB per step)",
                         parallelism=f"layer-sharded x{world}, no collective"),
@@ -319,9 +323,19 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-steps", type=int, default=24)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: use only this many of the workload's layers")
+    ap.add_argument("--max-removed", type=int, default=0,
+                    help="profiling aid: stop the greedy loop after this many removals")
+    ap.add_argument("--skip-e2e", action="store_true", help="profiling aid: no host-buffer leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     shape = wl.CONFIGS[WORKLOAD][0]
+    if args.layers > 0:
+        shape = wl.scaled(shape, n_layers=args.layers)
+    if args.max_removed > 0:
+        keep = shape.n_groups - args.max_removed
+        shape = wl.scaled(shape, levels=tuple(v for v in shape.levels if v > keep) + (keep,))
     if args.impl == "reference":
         run_reference(args, shape)
     else:
