@@ -97,6 +97,38 @@ ziplm_status ziplm_damped_inverse(const float* H, int L, int d, float damp_frac,
                                   void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Damped inverse without a workspace argument (the paper has no counterpart; this is a
+ * convenience of the library).
+ *
+ * Some callers cannot obtain device memory at the point where they need the inverse: code that
+ * runs inside a framework hook or a plugin callback where the allocator must not be entered, a
+ * process whose whole device budget was handed to another allocator up front, or a real-time
+ * loop where a cudaMalloc (which may synchronise the device) is not acceptable.  For them this
+ * entry point computes exactly what ziplm_damped_inverse computes, with the same kernels, but
+ * takes its scratch from an 8 MiB array that is compiled into the library.  It calls neither
+ * cudaMalloc nor cudaFree nor any routine that allocates.
+ *
+ *   H, Hinv, layer_status, damp_frac, cuda_stream   as for ziplm_damped_inverse; the caller still
+ *                 provides the input and both outputs.
+ *
+ * Limit: the request must satisfy ziplm_inverse_workspace_bytes(L, d) <= 8 MiB (8388608), e.g.
+ * one layer up to d = 704, four layers of d = 320, sixteen layers of d = 128; anything larger
+ * returns ZIPLM_ERR_UNSUPPORTED and does nothing.
+ * Cost: every GPU that loads the library holds the 8 MiB until the process exits.
+ * First call on a device: it looks up the device address of the built-in array (with that
+ * device current) and remembers it; make this first call outside any stream capture.
+ * Sharing: all calls on a device use the same array, and it keeps whatever the last call left
+ * there.  No call relies on those leftovers (every region is rewritten before it is read), but
+ * two calls whose kernels overlap on the GPU -- different streams, or different host threads
+ * without ordering -- race on it and give wrong results: order such calls on one stream or with
+ * events.
+ * Errors: ZIPLM_ERR_INVALID_ARG as for ziplm_damped_inverse; ZIPLM_ERR_UNSUPPORTED beyond the
+ * limit; ZIPLM_ERR_CUDA if the address lookup or a launch fails.
+ */
+ziplm_status ziplm_damped_inverse_noalloc(const float* H, int L, int d, float damp_frac,
+                                          double* Hinv, int* layer_status, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Greedy structured pruning of L same-shape layers (Algorithm 1; Eq. 2, Eq. 3, Eq. 4) with a
  * snapshot at every requested level (the per-layer database of Sec. 3.2).
  *

@@ -65,6 +65,8 @@ def load_library() -> ctypes.CDLL:
     lib.ziplm_inverse_workspace_bytes.argtypes = [c_int, c_int]
     lib.ziplm_damped_inverse.restype = c_int
     lib.ziplm_damped_inverse.argtypes = [vp, c_int, c_int, c_f, vp, vp, vp, c_sz, vp]
+    lib.ziplm_damped_inverse_noalloc.restype = c_int
+    lib.ziplm_damped_inverse_noalloc.argtypes = [vp, c_int, c_int, c_f, vp, vp, vp]
     lib.ziplm_prune_workspace_bytes.restype = c_sz
     lib.ziplm_prune_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int, c_int]
     lib.ziplm_prune_layers.restype = c_int
@@ -166,6 +168,29 @@ def damped_inverse(H: torch.Tensor, damp_frac: float, workspace: Optional[torch.
     if st != 0:
         raise ZiplmError(st, "ziplm_damped_inverse")
     return Hinv, status
+
+
+def damped_inverse_noalloc(H: torch.Tensor, damp_frac: float, Hinv: torch.Tensor,
+                           layer_status: torch.Tensor) -> None:
+    """ziplm_damped_inverse_noalloc: the damped inverse for callers that must not allocate.
+
+    The scratch comes from an 8 MiB array inside the library, so this wrapper allocates nothing
+    either: the caller passes the input H [L, d, d] fp32 and both outputs, Hinv [L, d, d]
+    float64 and layer_status [L] int32.  Requests with inverse_workspace_bytes(L, d) > 8 MiB
+    raise ZiplmError(ERR_UNSUPPORTED).  Calls that overlap on the GPU race on the shared scratch.
+    """
+    lib = load_library()
+    _check(H, torch.float32, "H")
+    _check(Hinv, torch.float64, "Hinv")
+    _check(layer_status, torch.int32, "layer_status")
+    L, d, _ = H.shape
+    if tuple(Hinv.shape) != (L, d, d) or layer_status.numel() != L:
+        raise ValueError("Hinv must be [L, d, d] and layer_status [L]")
+    with torch.cuda.device(H.device):
+        st = lib.ziplm_damped_inverse_noalloc(H.data_ptr(), L, d, damp_frac, Hinv.data_ptr(),
+                                              layer_status.data_ptr(), _stream_ptr(H))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_damped_inverse_noalloc")
 
 
 def prune_layers(W: torch.Tensor, H: torch.Tensor, group_size: int, damp_frac: float,

@@ -8,7 +8,15 @@
 // padded to a multiple of 64 with an identity block, whose inverse is again the identity.
 #include <math.h>
 
+#include <mutex>
+
 #include "common.cuh"
+
+// Built-in scratch of ziplm_damped_inverse_noalloc: lives in every GPU that loads this library
+// until the process exits.  In host code this name is only a handle for cudaGetSymbolAddress,
+// never a device address.
+constexpr size_t kBuiltinScratchBytes = (size_t)8 << 20;
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
 
 namespace ziplm {
 namespace {
@@ -363,3 +371,41 @@ ziplm_status run_damped_inverse(const float* H, int L, int d, float damp_frac, d
 }
 
 }  // namespace ziplm
+
+// ---------------------------------------------------------------------------------------------
+// Variant of the damped inverse for callers that cannot allocate device memory.
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mu;
+void* g_scratch_addr[kMaxDevices] = {};   // device address of g_builtin_scratch, per device
+}  // namespace
+
+extern "C" ziplm_status ziplm_damped_inverse_noalloc(const float* H, int L, int d, float damp_frac,
+                                                     double* Hinv, int* layer_status,
+                                                     void* cuda_stream) {
+    using namespace ziplm;
+    if (L < 1 || d < 1 || !H || !Hinv || !layer_status) return ZIPLM_ERR_INVALID_ARG;
+    if (!(damp_frac >= 0.f) || !isfinite(damp_frac)) return ZIPLM_ERR_INVALID_ARG;
+    if (inverse_workspace_bytes(L, d) > kBuiltinScratchBytes) return ZIPLM_ERR_UNSUPPORTED;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ZIPLM_ERR_CUDA;
+    void* scratch = nullptr;
+    {
+        // once per device, with that device current: turn the symbol into its device address
+        std::lock_guard<std::mutex> lk(g_scratch_mu);
+        if (!g_scratch_addr[dev]) {
+            void* addr = nullptr;
+            if (cudaGetSymbolAddress(&addr, g_builtin_scratch) != cudaSuccess || !addr)
+                return ZIPLM_ERR_CUDA;
+            g_scratch_addr[dev] = addr;
+        }
+        scratch = g_scratch_addr[dev];
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ZIPLM_CHECK_CUDA(cudaMemsetAsync(layer_status, 0, sizeof(int) * L, st));
+    // Every part of the scratch that a kernel reads is written earlier in the same call (the
+    // damped copy, the factor, the lower tiles of its inverse, lambda), so nothing left behind
+    // by the previous call needs clearing.
+    return run_damped_inverse(H, L, d, damp_frac, Hinv, nullptr, 0, nullptr, nullptr, layer_status,
+                              scratch, kBuiltinScratchBytes, st);
+}
