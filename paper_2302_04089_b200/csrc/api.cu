@@ -1,6 +1,7 @@
 // extern "C" boundary: argument validation and dispatch.  No device memory is allocated here and
 // nothing synchronises; every stage is enqueued on the caller's stream.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -9,6 +10,13 @@ using namespace ziplm;
 namespace {
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Debugging switch: ZIPLM_FORCE_BLOCK_PATH=1 sends group_size 1 through the general block path
+// (float64 state, g x g Cholesky per structure) instead of the streaming neuron path.
+bool force_block_path() {
+    const char* e = getenv("ZIPLM_FORCE_BLOCK_PATH");
+    return e && e[0] == '1';
+}
 
 bool have_device() {
     int dev = -1;
@@ -80,7 +88,8 @@ ziplm_status ziplm_damped_inverse(const float* H, int L, int d, float damp_frac,
 size_t ziplm_prune_workspace_bytes(int L, int d_row, int d_col, int group_size, int n_levels) {
     if (L < 1 || d_row < 1 || d_col < 1 || group_size < 1 || n_levels < 0) return 0;
     if (d_col % group_size != 0 || group_size > 64) return 0;
-    if (group_size == 1) return neuron_workspace_bytes(L, d_row, d_col, n_levels);
+    if (group_size == 1 && !force_block_path())
+        return neuron_workspace_bytes(L, d_row, d_col, n_levels);
     return block_workspace_bytes(L, d_row, d_col, group_size, n_levels);
 }
 
@@ -105,7 +114,7 @@ ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row
     if (!have_device()) return ZIPLM_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     ZIPLM_CHECK_CUDA(cudaMemsetAsync(layer_status, 0, sizeof(int) * L, st));
-    if (group_size == 1)
+    if (group_size == 1 && !force_block_path())
         return run_prune_neurons(W, H, L, d_row, d_col, damp_frac, levels, n_levels, W_snap, loss,
                                  base_loss, order, saliency, layer_status, workspace,
                                  workspace_bytes, st);

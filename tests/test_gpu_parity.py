@@ -170,6 +170,43 @@ def test_workspace_is_not_assumed_clean():
         compare_layer(W[l].numpy(), H[l].numpy(), 1, 0.01, [50, 10], out, l)
 
 
+# ------------------------------------------------------------------ block path (a4', heads)
+@pytest.mark.parametrize("d,g,r,L,levels", [
+    (256, 64, 64, 2, [4, 3, 2, 1, 0]),          # four heads, every head count
+    (96, 2, 20, 2, [48, 40, 17, 0]),            # tiny groups, many steps
+    (120, 24, 33, 1, [4, 1]),                   # group size that is no power of two, ragged rows
+    (192, 64, 200, 3, [2]),
+])
+def test_block_path_small_shapes(d, g, r, L, levels):
+    sh = wl.scaled(wl.CONFIGS["c2_bert_base_attn"][0], d_col=d, d_row=r, group_size=g,
+                   n_tokens=4 * d + 16, n_layers=L, levels=tuple(levels))
+    run_case(sh)
+
+
+def test_c2_bert_base_attention_shape_three_layers():
+    """Full-size attention out-projection (768 x 768, 12 heads x 64), 3 of the 12 layers."""
+    sh = wl.CONFIGS["c2_bert_base_attn"][0]
+    run_case(sh, layers=[0, 5, 11])
+
+
+def test_block_path_with_group_size_one_agrees_with_neuron_path(monkeypatch):
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=128, d_row=40, d_latent=32,
+                   n_tokens=600, n_layers=2, levels=(128, 64, 0))
+    W, X = wl.make_layers(sh, "cpu")
+    H = torch.stack([oracle_h32(X[l]) for l in range(2)])
+    a = z.prune_layers(W.cuda(), H.cuda(), 1, 0.01, [128, 64, 0])
+    monkeypatch.setenv("ZIPLM_FORCE_BLOCK_PATH", "1")
+    b = z.prune_layers(W.cuda(), H.cuda(), 1, 0.01, [128, 64, 0])
+    torch.cuda.synchronize()
+    monkeypatch.delenv("ZIPLM_FORCE_BLOCK_PATH")
+    assert torch.equal(a["order"], b["order"])
+    assert torch.allclose(a["W_snap"], b["W_snap"], rtol=1e-4, atol=1e-7)
+    assert torch.allclose(a["loss"], b["loss"], rtol=1e-4)
+    for l in range(2):
+        compare_layer(W[l].numpy(), H[l].numpy(), 1, 0.01, [128, 64, 0], b, l)
+
+
 # ------------------------------------------------------------------ host-side argument checks
 def test_invalid_arguments_are_rejected_on_the_host():
     z = zb()
