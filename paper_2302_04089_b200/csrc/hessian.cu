@@ -3,10 +3,14 @@
 // K-major tiles of the same matrix; only tiles on or below the diagonal are computed and the
 // result is mirrored (symmetric rank-k update).
 //
-// This file holds the CUDA-core route: fp32 FMA on 64 x 64 tiles with a two-level fp32 sum (the
-// running tile sum is folded into a second accumulator every 512 tokens, which keeps the
-// rounding error of a 1e4 .. 1e5 term sum near the fp32 unit roundoff).
+// This file holds the route choice and the CUDA-core route: fp32 FMA on 64 x 64 tiles with a
+// two-level fp32 sum (the running tile sum is folded into a second accumulator every 512 tokens,
+// which keeps the rounding error of a 1e4 .. 1e5 term sum near the fp32 unit roundoff).  The
+// tensor-core route (hessian_tc.cu) is the default; the CUDA-core route serves token counts
+// below one K block and can be forced with ZIPLM_HESSIAN_ROUTE=simt for comparison.
 #include <cuda_bf16.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 
@@ -113,17 +117,22 @@ __global__ void k_scale_h(float* __restrict__ H, size_t count, float beta) {
     if (i < count) H[i] = (beta == 0.f) ? 0.f : H[i] * beta;
 }
 
+bool use_tensor_cores(long long N) {
+    const char* e = getenv("ZIPLM_HESSIAN_ROUTE");
+    if (e && strcmp(e, "simt") == 0) return false;
+    if (e && strcmp(e, "tc") == 0) return N > 0;
+    return N >= 32;
+}
+
 }  // namespace
 
 size_t hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt) {
-    (void)L; (void)d; (void)n_tokens; (void)dt;
-    return 0;
+    return use_tensor_cores(n_tokens) ? hessian_tc_workspace_bytes(L, d, n_tokens, dt) : 0;
 }
 
 ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, int L, int d, long long N,
                          long long ldx, float alpha, float beta, void* ws, size_t ws_bytes,
                          cudaStream_t st) {
-    (void)ws; (void)ws_bytes;
     if (N == 0) {
         const size_t count = (size_t)L * d * d;
         if (beta != 1.f) {
@@ -132,6 +141,8 @@ ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, int L, int d, 
         }
         return ZIPLM_OK;
     }
+    if (use_tensor_cores(N))
+        return run_hessian_tc(H, X, dt, L, d, N, ldx, alpha, beta, ws, ws_bytes, st);
     const int T = (d + 63) / 64;
     const dim3 grid(T * (T + 1) / 2, L);
     if (dt == ZIPLM_F32)
