@@ -11,8 +11,8 @@
 //            and X_lo = X - X_hi; the kernel accumulates hi*hi + hi*lo + lo*hi with kind::tf32,
 //            which keeps ~21 mantissa bits per product.  K block of 32 tokens.
 //
-// One CTA per tile: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 =
-// epilogue (one TMEM lane quarter each; they drain the accumulator every few K blocks, see
+// One CTA per tile: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..9 =
+// epilogue (two per TMEM lane quarter; they drain the accumulator every few K blocks, see
 // below).  Every mbarrier wait is bounded; if one runs out the
 // kernel raises the error word, poisons H[l][0][0] with NaN and leaves through the normal exit
 // (TMEM freed), so a lost copy can never hang the GPU.
@@ -119,18 +119,23 @@ __host__ __device__ constexpr uint32_t make_idesc(uint32_t fmt) {
 
 // Tensor-memory accumulators truncate when they add (measured: the error of a chain of S
 // accumulating MMAs grows like S * 3e-8, always toward zero), so a chain is kept short: the main
-// accumulator is double-buffered, and after every CHUNK K blocks (16 MMAs) the epilogue warps
-// drain it into fp32 registers, where the partial sums are added with round-to-nearest.  The
-// TF32 cross terms hi*lo + lo*hi are 2^-11 of the main term; they get an accumulator of their
-// own that is only read at the end, so their truncation is negligible.
-constexpr int CHUNK = 4;
+// accumulator is double-buffered, and after every CHUNK K blocks (8 MMAs) the epilogue warps
+// drain it into fp32 registers, where the partial sums are added with round-to-nearest in two
+// levels (a running sum that is folded into the total every FOLD drains, so that neither level
+// adds more than a few dozen terms).  The TF32 cross terms hi*lo + lo*hi are 2^-11 of the main
+// term; they get an accumulator of their own that is only read at the end, so their truncation
+// is negligible.
+constexpr int CHUNK = 2;
+constexpr int FOLD = 32;
+constexpr int EPI_WARPS = 8;                  // two warps per TMEM lane quarter, 64 columns each
+constexpr int THREADS = 32 * (2 + EPI_WARPS);
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 template <bool TF32>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(THREADS, 1)
 k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
           float* __restrict__ H, int d, int num_kb, float alpha, float beta, int layer0,
           int* __restrict__ err_word) {
@@ -161,7 +166,7 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_acc_full[b]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[b]), 4);    // one arrival per epilogue warp
+            mbar_init(smem_u32(&bar_acc_empty[b]), EPI_WARPS);   // one arrival per epilogue warp
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -242,12 +247,14 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
             }
         }
     } else {
-        // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4
+        // ---------------- epilogue: warps 2..9; TMEM lane quarter = warp % 4, column half by warp
         const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-        float acc[TM];
+        constexpr int NC = TM / 2;                      // columns owned by this thread
+        float acc[NC], tot[NC];
 #pragma unroll
-        for (int e = 0; e < TM; ++e) acc[e] = 0.f;
+        for (int e = 0; e < NC; ++e) { acc[e] = 0.f; tot[e] = 0.f; }
         for (int c = 0; c < num_chunks; ++c) {
             const int b = c & 1;
             if (!mbar_wait(smem_u32(&bar_acc_full[b]), ((uint32_t)c >> 1) & 1u, abortp)) failed = true;
@@ -255,23 +262,27 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
             if (failed) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-            for (int cc = 0; cc < TM / 32; ++cc) {
+            for (int cc = 0; cc < NC / 32; ++cc) {
                 uint32_t v[32];
-                tmem_ld32(tmem_base + lane_base + (uint32_t)(b * 128 + cc * 32), v);
+                tmem_ld32(tmem_base + lane_base + (uint32_t)(b * 128 + half * NC + cc * 32), v);
 #pragma unroll
                 for (int e = 0; e < 32; ++e) acc[cc * 32 + e] += __uint_as_float(v[e]);
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[b]));
+            if ((c % FOLD) == FOLD - 1) {
+#pragma unroll
+                for (int e = 0; e < NC; ++e) { tot[e] += acc[e]; acc[e] = 0.f; }
+            }
         }
         if (!failed) {
             if (TF32) {
                 // the last chunk's commit also covers every cross-term MMA
 #pragma unroll
-                for (int cc = 0; cc < TM / 32; ++cc) {
+                for (int cc = 0; cc < NC / 32; ++cc) {
                     uint32_t v[32];
-                    tmem_ld32(tmem_base + lane_base + (uint32_t)(256 + cc * 32), v);
+                    tmem_ld32(tmem_base + lane_base + (uint32_t)(256 + half * NC + cc * 32), v);
 #pragma unroll
                     for (int e = 0; e < 32; ++e) acc[cc * 32 + e] += __uint_as_float(v[e]);
                 }
@@ -279,9 +290,9 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
             float* Hl = H + (size_t)(layer0 + l) * d * d;
             const int row = i0 + q * 32 + lane;
 #pragma unroll
-            for (int e = 0; e < TM; ++e) {
-                const int col = j0 + e;
-                float val = alpha * acc[e];
+            for (int e = 0; e < NC; ++e) {
+                const int col = j0 + half * NC + e;
+                float val = alpha * (tot[e] + acc[e]);
                 if (row < d && col < d && col <= row) {
                     if (beta != 0.f) val += Hl[(size_t)row * d + col];
                     Hl[(size_t)row * d + col] = val;
@@ -435,7 +446,7 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, int L, int 
             CUtensorMap mh, ml;
             if (!make_map(&mh, hi, true, N, d, ln, np) || !make_map(&ml, lo, true, N, d, ln, np))
                 return ZIPLM_ERR_CUDA;
-            k_syrk_tc<true><<<dim3(n_tiles, ln), 192, smem_tf32, st>>>(mh, ml, H, d, num_kb, alpha, beta,
+            k_syrk_tc<true><<<dim3(n_tiles, ln), THREADS, smem_tf32, st>>>(mh, ml, H, d, num_kb, alpha, beta,
                                                                       l0, err_word);
             ZIPLM_CHECK_LAUNCH();
         }
@@ -448,7 +459,7 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, int L, int 
             CUtensorMap mx;
             const __nv_bfloat16* Xc = static_cast<const __nv_bfloat16*>(X) + (size_t)l0 * d * ldx;
             if (!make_map(&mx, Xc, false, N, d, ln, ldx)) return ZIPLM_ERR_CUDA;
-            k_syrk_tc<false><<<dim3(n_tiles, ln), 192, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
+            k_syrk_tc<false><<<dim3(n_tiles, ln), THREADS, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
                                                                        l0, err_word);
             ZIPLM_CHECK_LAUNCH();
         }
