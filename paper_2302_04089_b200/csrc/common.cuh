@@ -82,6 +82,14 @@ ziplm_status run_prune_neurons(const float* W, const float* H, int L, int r, int
                                float* loss, float* base_loss, int* order, float* saliency,
                                int* layer_status, void* ws, size_t ws_bytes, cudaStream_t st);
 
+// Neuron path with delayed rank-B updates (prune_lazy.cu); chosen by run_prune_neurons.
+bool lazy_path_supported(int d);
+size_t lazy_workspace_bytes(int L, int r, int d, int n_levels);
+ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d, float damp_frac,
+                            const int* levels, int n_levels, float* W_snap, float* loss,
+                            float* base_loss, int* order, float* saliency, int* layer_status,
+                            void* ws, size_t ws_bytes, cudaStream_t st);
+
 size_t block_workspace_bytes(int L, int r, int d, int g, int n_levels);
 ziplm_status run_prune_blocks(const float* W, const float* H, int L, int r, int d, int g,
                               float damp_frac, const int* levels, int n_levels, float* W_snap,

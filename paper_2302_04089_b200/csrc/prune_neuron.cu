@@ -23,6 +23,8 @@
 // Algorithm 1 -- so they are simply dropped).  The live problem is therefore always the leading
 // n x n corner, and every step streams exactly the live bytes.
 #include <math.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 
@@ -374,9 +376,18 @@ NeuronWs carve_neuron(void* ws, int L, int r, int d) {
 
 }  // namespace
 
+// The delayed-update variant (prune_lazy.cu) is the default where it applies; the streaming
+// variant in this file serves the other shapes and ZIPLM_NEURON_PATH=stream selects it always.
+static bool use_lazy_path(int d) {
+    const char* e = getenv("ZIPLM_NEURON_PATH");
+    if (e && strcmp(e, "stream") == 0) return false;
+    return lazy_path_supported(d);
+}
+
 size_t neuron_workspace_bytes(int L, int r, int d, int n_levels) {
-    (void)n_levels;
-    return carve_neuron(nullptr, L, r, d).total;
+    const size_t a = carve_neuron(nullptr, L, r, d).total;
+    const size_t b = lazy_path_supported(d) ? lazy_workspace_bytes(L, r, d, n_levels) : 0;
+    return a > b ? a : b;
 }
 
 ziplm_status run_prune_neurons(const float* W, const float* H, int L, int r, int d,
@@ -384,6 +395,9 @@ ziplm_status run_prune_neurons(const float* W, const float* H, int L, int r, int
                                float* loss, float* base_loss, int* order, float* saliency,
                                int* layer_status, void* ws, size_t ws_bytes, cudaStream_t st) {
     if (ws_bytes < neuron_workspace_bytes(L, r, d, n_levels)) return ZIPLM_ERR_WORKSPACE;
+    if (use_lazy_path(d))
+        return run_prune_lazy(W, H, L, r, d, damp_frac, levels, n_levels, W_snap, loss, base_loss,
+                              order, saliency, layer_status, ws, ws_bytes, st);
     NeuronWs w = carve_neuron(ws, L, r, d);
     const int G = d;
 

@@ -118,7 +118,18 @@ def test_not_positive_definite_layer_is_flagged_and_others_finish():
 
 
 # ------------------------------------------------------------------ neuron path (a4 - a10)
-def test_c1_tiny_ffn_full_config():
+@pytest.fixture(params=["lazy", "stream"])
+def neuron_path(request, monkeypatch):
+    """Run a test once per neuron-path variant: delayed rank-B updates (default where the shape
+    allows it) and the per-step streaming update."""
+    if request.param == "stream":
+        monkeypatch.setenv("ZIPLM_NEURON_PATH", "stream")
+    else:
+        monkeypatch.delenv("ZIPLM_NEURON_PATH", raising=False)
+    return request.param
+
+
+def test_c1_tiny_ffn_full_config(neuron_path):
     out, reports = run_case(wl.CONFIGS["c1_tiny_ffn"][0])
     assert reports[0]["steps"] == 192
 
@@ -128,14 +139,16 @@ def test_c1_tiny_ffn_full_config():
     (64, 7, 1, [63, 0]),
     (130, 129, 3, [65]),
     (8, 4, 2, [4]),
+    (132, 30, 2, [132, 100, 99, 35, 3, 0]),    # multiple of 4: both variants; uneven block lengths
+    (4, 3, 1, [3, 2, 1, 0]),
 ])
-def test_neuron_path_ragged_shapes(d, r, L, levels):
+def test_neuron_path_ragged_shapes(d, r, L, levels, neuron_path):
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=d, d_row=r, d_latent=max(4, d // 4),
                    n_tokens=4 * d + 8, n_layers=L, levels=tuple(levels))
     run_case(sh)
 
 
-def test_neuron_path_mid_size_full_depth_three_layers():
+def test_neuron_path_mid_size_full_depth_three_layers(neuron_path):
     """Scaled BERT-base fc2: several row blocks per step, full greedy order 768 -> 0."""
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=768, d_row=192, d_latent=192,
                    n_tokens=4096, n_layers=3, levels=tuple(range(704, -1, -64)))
@@ -143,7 +156,7 @@ def test_neuron_path_mid_size_full_depth_three_layers():
     print(reports)
 
 
-def test_neuron_path_is_deterministic():
+def test_neuron_path_is_deterministic(neuron_path):
     z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=256, d_row=64, d_latent=64,
                    n_tokens=1024, n_layers=2, levels=(128, 0))
@@ -156,7 +169,7 @@ def test_neuron_path_is_deterministic():
     assert torch.equal(a["W_snap"], b["W_snap"])
 
 
-def test_workspace_is_not_assumed_clean():
+def test_workspace_is_not_assumed_clean(neuron_path):
     """Poison the workspace with NaN bit patterns: values of unused slots never feed live ones."""
     z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=100, d_row=20, d_latent=25,
@@ -189,7 +202,7 @@ def test_c2_bert_base_attention_shape_three_layers():
     run_case(sh, layers=[0, 5, 11])
 
 
-def test_block_path_with_group_size_one_agrees_with_neuron_path(monkeypatch):
+def test_block_path_with_group_size_one_agrees_with_neuron_path(monkeypatch, neuron_path):
     z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=128, d_row=40, d_latent=32,
                    n_tokens=600, n_layers=2, levels=(128, 64, 0))
