@@ -167,6 +167,32 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 # CUDA leg
 # ------------------------------------------------------------------------------------------
+LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in prune_lazy.cu)
+
+
+def lazy_update_work(L, G, levels):
+    """Algorithmic work of k_lazy_update_aq over one greedy run: a launch that leaves n live
+    structures reads and writes the strict lower triangles of H^-1 and Q once (2 matrices x
+    n(n-1)/2 entries x 4 B x (read + write)) and spends 3 fp32 FMA per entry and pending step.
+    Block boundaries fall on the requested levels, as in the library.  Returns (bytes, fma,
+    launches)."""
+    n, slot, nbytes, fma, launches = G, 0, 0.0, 0.0, 0
+    levels = [v for v in levels if v < G]
+    n_min = levels[-1] if levels else G
+    while n > n_min:
+        stop = levels[slot] if slot < len(levels) else n_min
+        m = min(LAZY_BLOCK, n - stop)
+        n -= m
+        if n > 1:
+            entries = L * n * (n - 1) / 2.0
+            nbytes += 16.0 * entries
+            fma += 3.0 * m * entries
+            launches += 1
+        if slot < len(levels) and levels[slot] == n:
+            slot += 1
+    return nbytes, fma, launches
+
+
 def update_bytes(L, r, G, n_removed):
     """Algorithmic bytes of the fused H^-1 / W update over the whole greedy loop: per launch
     with n live structures, L * (8 r n + 4 n^2) (read + write of the live W, read + write of one
@@ -263,11 +289,19 @@ def run_ours(args, shape):
         barrier()
         ms_e2e = e0.elapsed_time(e1) / e2e_steps
 
-    # ---- one more step with per-phase event timing (roofline of the update kernel)
+    # ---- one more step with per-phase event timing (roofline of the dominant kernel), and one
+    # with the per-step streaming update selected, whose fused H^-1 / W kernel is reported too
     z.profile_begin()
     step()
     torch.cuda.synchronize()
     phases = z.profile_end()
+    os.environ["ZIPLM_NEURON_PATH"] = "stream"
+    step()
+    z.profile_begin()
+    step()
+    torch.cuda.synchronize()
+    phases_stream = z.profile_end()
+    del os.environ["ZIPLM_NEURON_PATH"]
 
     if dist is not None:
         t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
@@ -280,9 +314,13 @@ def run_ours(args, shape):
 
     if rank == 0:
         peak, peak_src = load_peaks()
-        upd_ms, upd_n = phases["update"]
+        upd_ms, upd_n = phases_stream["update"]
         alg_bytes, n_launch = update_bytes(L, r, G, n_removed)
         achieved = alg_bytes / (upd_ms * 1e-3) / 1e9 if upd_ms > 0 else 0.0
+        aq_ms, aq_n = phases.get("lazy_update_aq", (0.0, 0))
+        aq_bytes, aq_fma, _ = lazy_update_work(L, G, levels)
+        aq_gbs = aq_bytes / (aq_ms * 1e-3) / 1e9 if aq_ms > 0 else 0.0
+        fma_peak = 148 * 128 * 1.965e9 / 1e12          # fp32 TFMA/s: SMs x lanes x max SM clock
         line = dict(
             metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
             warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
@@ -298,10 +336,21 @@ def run_ours(args, shape):
                      ms_per_step=ms_e2e),
             gpu_launches=int(launches),
             clocks=clocks,
-            roofline=dict(kernel="k_neuron_update", bound="hbm", achieved=achieved, peak=peak,
-                          unit="GB/s", frac=achieved / peak, traffic=None, peak_source=peak_src,
-                          launches=upd_n, avg_launch_us=1e3 * upd_ms / max(upd_n, 1),
-                          algorithmic_bytes_per_step=alg_bytes),
+            roofline=dict(kernel="k_lazy_update_aq", bound="hbm", achieved=aq_gbs, peak=peak,
+                          unit="GB/s", frac=aq_gbs / peak, traffic=None, peak_source=peak_src,
+                          launches=aq_n, avg_launch_us=1e3 * aq_ms / max(aq_n, 1),
+                          algorithmic_bytes_per_step=aq_bytes,
+                          alu=dict(achieved_tfma=aq_fma / (aq_ms * 1e-3) / 1e12 if aq_ms > 0 else 0.0,
+                                   peak_tfma=fma_peak,
+                                   note="3 fp32 FMA per entry and pending step; peak = 148 SMs x "
+                                        "128 lanes x 1.965 GHz")),
+            roofline_streaming_update=dict(
+                kernel="k_neuron_update", bound="hbm", achieved=achieved, peak=peak, unit="GB/s",
+                frac=achieved / peak, traffic=None, peak_source=peak_src, launches=upd_n,
+                avg_launch_us=1e3 * upd_ms / max(upd_n, 1), algorithmic_bytes_per_step=alg_bytes,
+                note="per-step fused H^-1/W update of the streaming variant "
+                     "(ZIPLM_NEURON_PATH=stream), timed in a separate step",
+                phases_ms={k: round(v[0], 3) for k, v in phases_stream.items() if v[1] > 0}),
         )
         if world == 1 and not args.no_cpu_baseline:
             s = oracle_sample(shape, n_loop_steps=args.oracle_steps)

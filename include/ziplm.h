@@ -184,7 +184,7 @@ ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row
  *                          phase, the summed milliseconds (host [n_phases] double, may be NULL)
  *                          and the number of bracketed spans (host [n_phases], may be NULL).
  * ziplm_profile_phase_count / ziplm_profile_phase_name   enumerate the phases ("hessian",
- *                          "inverse", "init", "prep", "update", "snapshot", ...).
+ *                          "inverse", "init", "prep", "update", "snapshot", "lazy_steps", ...).
  */
 long long ziplm_launch_count(void);
 ziplm_status ziplm_profile_begin(void);

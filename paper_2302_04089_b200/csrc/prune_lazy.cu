@@ -447,6 +447,38 @@ __global__ void k_lazy_loss(int L, int n_levels, int slot, const double* __restr
     state[l].dw2 = 0.0;
 }
 
+// base_loss = ||W X||_F^2 = 1/2 tr(W H W^T) = 1/2 <W^T W, H>: one elementwise pass over the Gram
+// matrix (full symmetric right after the product kernel) and the undamped Hessian.
+__global__ void __launch_bounds__(256) k_lazy_base_loss(int d, const float* __restrict__ Q,
+                                                        const float* __restrict__ H,
+                                                        double* __restrict__ acc64) {
+    __shared__ double red[8];
+    const int l = blockIdx.y;
+    const size_t count = (size_t)d * d / 4;
+    const float4* q4 = reinterpret_cast<const float4*>(Q + (size_t)l * d * d);
+    const float4* h4 = reinterpret_cast<const float4*>(H + (size_t)l * d * d);
+    double acc = 0.0;
+    for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < count; e += (size_t)gridDim.x * 256) {
+        const float4 a = __ldg(q4 + e), b = __ldg(h4 + e);
+        acc += (double)a.x * b.x + (double)a.y * b.y + (double)a.z * b.z + (double)a.w * b.w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        atomicAdd(acc64 + l, t);
+    }
+}
+
+__global__ void k_lazy_base_finish(int L, const double* __restrict__ acc64,
+                                   float* __restrict__ base_loss) {
+    const int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l < L) base_loss[l] = (float)(0.5 * acc64[l]);
+}
+
 struct LazyWs {
     float* A[2]; float* Q[2]; float* Wt[2];
     double* dA[2]; double* dQ[2]; int* idx[2];
@@ -518,7 +550,13 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
         ziplm_status g = run_hessian_tc(w.Q[0], w.Wt[0], ZIPLM_F32, L, d, rp, rp, 1.0f, 0.0f, w.aux,
                                         w.aux_bytes, st);
         if (g != ZIPLM_OK) return g;
-        if (base_loss) return run_base_loss(W, H, L, r, d, w.base_acc, base_loss, st);
+        if (base_loss) {
+            ZIPLM_CHECK_CUDA(cudaMemsetAsync(w.base_acc, 0, sizeof(double) * L, st));
+            k_lazy_base_loss<<<dim3(148, L), 256, 0, st>>>(d, w.Q[0], H, w.base_acc);
+            ZIPLM_CHECK_LAUNCH();
+            k_lazy_base_finish<<<(L + 63) / 64, 64, 0, st>>>(L, w.base_acc, base_loss);
+            ZIPLM_CHECK_LAUNCH();
+        }
         return ZIPLM_OK;
     };
     s = init();
@@ -548,7 +586,7 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
         const int nsteps = (n - stop < BMAX) ? (n - stop) : BMAX;
         const int nxt = cur ^ 1;
         {
-            PhaseScope ps(PH_PREP, st);
+            PhaseScope ps(PH_LAZY_STEPS, st);
             k_lazy_steps<<<L, STEP_THREADS, 0, st>>>(n, t, nsteps, d, G, r, rp, w.A[cur], w.Q[cur],
                                                     w.Wt[cur], w.dA[cur], w.dQ[cur], w.idx[cur],
                                                     w.dA[nxt], w.dQ[nxt], w.idx[nxt], w.src, w.U, w.Z,
@@ -556,14 +594,17 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
             ZIPLM_CHECK_LAUNCH();
         }
         const int n_new = n - nsteps;
-        if (n_new > 0) {
-            PhaseScope ps(PH_UPDATE, st);
-            if (n_new > 1) {
+        if (n_new > 1) {
+            PhaseScope ps(PH_LAZY_UPDATE_AQ, st);
+            {
                 const int T = (n_new + 63) / 64;
                 k_lazy_update_aq<<<dim3(T * (T + 1) / 2, L), 256, 0, st>>>(
                     n_new, nsteps, d, w.A[cur], w.Q[cur], w.A[nxt], w.Q[nxt], w.src, w.U, w.Z);
                 ZIPLM_CHECK_LAUNCH();
             }
+        }
+        if (n_new > 0) {
+            PhaseScope ps(PH_LAZY_UPDATE_W, st);
             k_lazy_update_w<<<dim3((n_new + 7) / 8, L), 256, 0, st>>>(n_new, nsteps, d, rp, w.Wt[cur],
                                                                      w.Wt[nxt], w.src, w.U, w.C);
             ZIPLM_CHECK_LAUNCH();
