@@ -18,13 +18,14 @@
 //     positions are squeezed out by a stable, out-of-place compaction, so the live problem is
 //     again the leading n x n corner in original column order.
 //
-// Launches per block, for all L layers at once: one "steps" kernel (one CTA per layer runs the
-// B greedy steps back to back with block-level barriers only -- layers are independent, so no
-// grid-wide synchronisation is needed) and two update kernels.  Block boundaries are placed on
+// Launches per block, for all L layers at once: one "steps" kernel (one thread-block cluster per
+// layer runs the B greedy steps back to back with one cluster barrier per step -- layers are
+// independent, so no grid-wide synchronisation is needed) and two update kernels.  Block boundaries are placed on
 // the requested levels, where W is up to date and can be snapshotted.
 //
 // Layout per layer: A, Q fp32 [d, d] strict lower triangles (two buffers each, ping-pong),
 // Wt = W^T fp32 [d, rp] (two buffers), float64 diagonals, pending U, Z [B, d] and C [B, rp].
+#include <cooperative_groups.h>
 #include <math.h>
 
 #include "common.cuh"
@@ -33,8 +34,9 @@ namespace ziplm {
 namespace {
 
 constexpr int BMAX = 32;         // pending steps per block
-constexpr int STEP_THREADS = 1024;
-constexpr int KPT = 4;           // positions per thread in the steps kernel: d <= 4096
+constexpr int STEP_THREADS = 256; // threads per CTA of the steps kernel, four positions each
+constexpr int SLICE_MAX = 768;   // positions per CTA: 2 * BMAX * SLICE_MAX * 4 B = 192 KiB of smem
+constexpr int CLUSTER_MAX = 8;   // portable cluster size
 
 struct LazyState {
     double sumrho;
@@ -108,21 +110,51 @@ __device__ __forceinline__ Cand shfl_cand(const Cand& c, int off) {
     return o;
 }
 
-// nsteps greedy steps of one layer per CTA, on the stale matrices plus the pending terms of this
-// block; then the stable compaction of the per-position vectors.
+__device__ __forceinline__ void merge_cand(Cand& best, const Cand& o) {
+    if (o.pos >= 0 && (best.pos < 0 || better(o, best))) best = o;
+}
+
+// nsteps greedy steps of one layer, run by a thread-block cluster of CS CTAs (CS = 1, 2, 4 or 8,
+// chosen so that a CTA's slice of positions fits its shared memory).  CTA `rank` owns the
+// positions [rank * S, rank * S + S); each of its 256 threads owns four consecutive ones and
+// keeps their float64 diagonal entries of H^-1 and Q in registers for the whole block.  The
+// pending vectors u_s, z_s of the block live in shared memory, sliced the same way, so the
+// correction of a pivot column touches no global memory; copies go to global memory only for
+// the update kernels that follow.  Per step there is one cluster barrier: every warp publishes
+// its best candidate, after the barrier warp 0 of every CTA reads all of them through
+// distributed shared memory and reaches the same pick, then fetches the pending vectors'
+// entries at the pivot from the CTA that owns it.
+// The scaled pivot columns of W (c_s) do not feed the selection; they are solved for at the end
+// of the block by forward substitution with the 32 x 32 triangle T[m][s] = u_s[p_m].
+// Finally the per-position vectors are compacted (stable) across the cluster.
 __global__ void __launch_bounds__(STEP_THREADS, 1)
-k_lazy_steps(int n0, int t0, int nsteps, int d, int G, int r, int rp, const float* __restrict__ A,
-             const float* __restrict__ Q, const float* __restrict__ Wt,
+k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
+             const float* __restrict__ A, const float* __restrict__ Q, const float* __restrict__ Wt,
              const double* __restrict__ dA_in, const double* __restrict__ dQ_in,
              const int* __restrict__ idx_in, double* __restrict__ dA_out,
              double* __restrict__ dQ_out, int* __restrict__ idx_out, int* __restrict__ src,
-             float* U, float* Z, float* C, LazyState* __restrict__ state, int* __restrict__ order,
-             float* __restrict__ saliency, int* layer_status) {
-    __shared__ Cand s_c[32];
+             float* __restrict__ U, float* __restrict__ Z, float* __restrict__ C,
+             LazyState* __restrict__ state, int* __restrict__ order, float* __restrict__ saliency,
+             int* layer_status) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int CS = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
+    const int l = blockIdx.x / CS;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int NW = STEP_THREADS / 32;
+
+    extern __shared__ float4 dyn_smem4[];
+    float* sU = reinterpret_cast<float*>(dyn_smem4);       // [BMAX][S]
+    float* sZ = sU + (size_t)BMAX * S;                     // [BMAX][S]
+    __shared__ Cand s_cand[2][NW];                         // per-warp candidates, by step parity
+    __shared__ float sT[BMAX][BMAX];                       // T[m][s] = u_s[p_m]
     __shared__ float sUp[BMAX], sZp[BMAX];
-    __shared__ int s_p, s_scan[32];
+    __shared__ int s_pm[BMAX];
+    __shared__ double s_rsm[BMAX];
+    __shared__ int s_p, s_count, s_wsum[NW];
     __shared__ double s_rs, s_half;
-    const int l = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
     const float* Al = A + (size_t)l * d * d;
     const float* Ql = Q + (size_t)l * d * d;
     const float* Wl = Wt + (size_t)l * d * rp;
@@ -130,144 +162,188 @@ k_lazy_steps(int n0, int t0, int nsteps, int d, int G, int r, int rp, const floa
     float* Zl = Z + (size_t)l * BMAX * d;
     float* Cl = C + (size_t)l * BMAX * rp;
 
-    double da[KPT], dq[KPT];
-    int org[KPT];
-    bool alive[KPT];
+    const int kloc = 4 * tid;                  // first owned position within the slice
+    const int k0 = rank * S + kloc;            // ... and globally
+    const bool owner_thread = (kloc < S) && (k0 < n0);
+    double da[4], dq[4];
+    int org[4];
+    bool alive[4];
 #pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const int k = tid + STEP_THREADS * j;
-        alive[j] = k < n0;
-        da[j] = alive[j] ? dA_in[(size_t)l * d + k] : 1.0;
-        dq[j] = alive[j] ? dQ_in[(size_t)l * d + k] : 0.0;
-        org[j] = alive[j] ? idx_in[(size_t)l * d + k] : 0x7fffffff;
+    for (int e = 0; e < 4; ++e) {
+        const int k = k0 + e;
+        alive[e] = owner_thread && k < n0;
+        da[e] = alive[e] ? dA_in[(size_t)l * d + k] : 1.0;
+        dq[e] = alive[e] ? dQ_in[(size_t)l * d + k] : 0.0;
+        org[e] = alive[e] ? idx_in[(size_t)l * d + k] : 0x7fffffff;
     }
+    double sumrho = 0.0;                       // meaningful in thread 0 of rank 0
 
     for (int m = 0; m < nsteps; ++m) {
-        // ---- argmin of rho = Q[k,k] / H^-1[k,k] over live positions (ties: lowest original index)
+        const int par = m & 1;
+        // ---- per-warp best of rho = Q[k,k] / H^-1[k,k] (ties: lowest original index)
         Cand best;
         best.rho = INFINITY; best.a = 1.0; best.q = 0.0; best.org = 0x7fffffff; best.pos = -1;
 #pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            if (!alive[j]) continue;
+        for (int e = 0; e < 4; ++e) {
+            if (!alive[e]) continue;
             Cand c;
-            c.rho = dq[j] / da[j];
+            c.rho = dq[e] / da[e];
             if (!(c.rho == c.rho)) c.rho = INFINITY;
-            c.a = da[j]; c.q = dq[j]; c.org = org[j]; c.pos = tid + STEP_THREADS * j;
-            if (best.pos < 0 || better(c, best)) best = c;
+            c.a = da[e]; c.q = dq[e]; c.org = org[e]; c.pos = k0 + e;
+            merge_cand(best, c);
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const Cand o = shfl_cand(best, off);
-            if (o.pos >= 0 && (best.pos < 0 || better(o, best))) best = o;
-        }
-        if (lane == 0) s_c[warp] = best;
-        __syncthreads();
+        for (int off = 16; off > 0; off >>= 1) merge_cand(best, shfl_cand(best, off));
+        if (lane == 0) s_cand[par][warp] = best;
+        cluster.sync();
+        // ---- warp 0 of every CTA: global pick from all warps of all CTAs, then the pending
+        //      vectors' entries at the pivot (from the CTA that owns it)
         if (warp == 0) {
-            best = s_c[lane];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const Cand o = shfl_cand(best, off);
-                if (o.pos >= 0 && (best.pos < 0 || better(o, best))) best = o;
+            Cand g;
+            g.rho = INFINITY; g.a = 1.0; g.q = 0.0; g.org = 0x7fffffff; g.pos = -1;
+            for (int e = lane; e < CS * NW; e += 32) {
+                const Cand* remote = cluster.map_shared_rank(&s_cand[par][e % NW], e / NW);
+                merge_cand(g, *remote);
             }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) merge_cand(g, shfl_cand(g, off));
+            int p = g.pos;
+            if (p < 0) p = 0;
+            double h = g.a;
+            int bad = 0;
+            if (!isfinite(g.rho) || !isfinite(h)) { bad = ZIPLM_ERR_NONFINITE; h = 1.0; }
+            else if (!(h > 0.0)) { bad = ZIPLM_ERR_NOT_PD; h = 1.0; }
+            const double rs = 1.0 / sqrt(h);
+            const int prow = p / S, pl = p - prow * S;
+            float up = 0.f, zp = 0.f;
+            if (lane < m) {
+                up = *cluster.map_shared_rank(sU + (size_t)lane * S + pl, prow);
+                zp = *cluster.map_shared_rank(sZ + (size_t)lane * S + pl, prow);
+            }
+            sUp[lane] = up;
+            sZp[lane] = zp;
+            sT[m][lane] = up;
             if (lane == 0) {
-                double h = best.a;
-                if (best.pos < 0) best.pos = 0;
-                if (!isfinite(best.rho) || !isfinite(h)) {
-                    set_layer_status(layer_status, l, ZIPLM_ERR_NONFINITE);
-                    h = 1.0;
-                } else if (!(h > 0.0)) {
-                    set_layer_status(layer_status, l, ZIPLM_ERR_NOT_PD);
-                    h = 1.0;
+                s_p = p;
+                s_rs = rs;
+                s_half = g.q / (2.0 * h);
+                s_pm[m] = p;
+                s_rsm[m] = rs;
+                if (rank == 0) {
+                    if (bad) set_layer_status(layer_status, l, bad);
+                    sumrho += isfinite(g.rho) ? g.rho : 0.0;
+                    order[(size_t)l * G + t0 + m] = g.org;
+                    if (saliency) saliency[(size_t)l * G + t0 + m] = (float)g.rho;
                 }
-                s_p = best.pos;
-                s_rs = 1.0 / sqrt(h);
-                s_half = best.q / (2.0 * h);
-                state[l].sumrho += isfinite(best.rho) ? best.rho : 0.0;
-                order[(size_t)l * G + t0 + m] = best.org;
-                if (saliency) saliency[(size_t)l * G + t0 + m] = (float)best.rho;
             }
         }
         __syncthreads();
         const int p = s_p;
         const double rs = s_rs, half = s_half;
-        // ---- values of the pending vectors at p
-        if (tid < m) {
-            sUp[tid] = Ul[(size_t)tid * d + p];
-            sZp[tid] = Zl[(size_t)tid * d + p];
-        }
-        __syncthreads();
-        // ---- true pivot columns of H^-1 and Q, float64 downdate of both diagonals
+        // ---- true pivot columns of H^-1 and Q on the owned positions; float64 diagonal downdate
+        if (owner_thread) {
+            double a[4], q[4];
 #pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            const int k = tid + STEP_THREADS * j;
-            if (k >= n0) continue;
-            float u32 = 0.f, z32 = 0.f;
-            if (alive[j] && k != p) {
-                const size_t off = (k < p) ? ((size_t)p * d + k) : ((size_t)k * d + p);
-                double a = (double)Al[off], q = (double)Ql[off];
-#pragma unroll 4
-                for (int s = 0; s < m; ++s) {
-                    const double us = (double)Ul[(size_t)s * d + k], zs = (double)Zl[(size_t)s * d + k];
-                    a = fma(-us, (double)sUp[s], a);
-                    q = fma(-zs, (double)sUp[s], q);
-                    q = fma(-us, (double)sZp[s], q);
+            for (int e = 0; e < 4; ++e) {
+                const int k = k0 + e;
+                a[e] = 0.0; q[e] = 0.0;
+                if (alive[e] && k != p) {
+                    const size_t off = (k < p) ? ((size_t)p * d + k) : ((size_t)k * d + p);
+                    a[e] = (double)Al[off];
+                    q[e] = (double)Ql[off];
                 }
-                const double u = a * rs;
-                const double z = q * rs - half * u;
-                da[j] -= u * u;
-                dq[j] -= 2.0 * z * u;
-                u32 = (float)u;
-                z32 = (float)z;
             }
-            if (k == p) alive[j] = false;
-            Ul[(size_t)m * d + k] = u32;
-            Zl[(size_t)m * d + k] = z32;
+            for (int s = 0; s < m; ++s) {
+                const float4 u4 = *reinterpret_cast<const float4*>(sU + (size_t)s * S + kloc);
+                const float4 z4 = *reinterpret_cast<const float4*>(sZ + (size_t)s * S + kloc);
+                const double up = (double)sUp[s], zp = (double)sZp[s];
+                const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, zz[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    a[e] = fma(-(double)uu[e], up, a[e]);
+                    q[e] = fma(-(double)zz[e], up, q[e]);
+                    q[e] = fma(-(double)uu[e], zp, q[e]);
+                }
+            }
+            float u32[4], z32[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int k = k0 + e;
+                u32[e] = 0.f; z32[e] = 0.f;
+                if (alive[e] && k != p) {
+                    const double u = a[e] * rs;
+                    const double z = q[e] * rs - half * u;
+                    da[e] -= u * u;
+                    dq[e] -= 2.0 * z * u;
+                    u32[e] = (float)u;
+                    z32[e] = (float)z;
+                }
+                if (k == p) alive[e] = false;
+            }
+            const float4 uo = make_float4(u32[0], u32[1], u32[2], u32[3]);
+            const float4 zo = make_float4(z32[0], z32[1], z32[2], z32[3]);
+            *reinterpret_cast<float4*>(sU + (size_t)m * S + kloc) = uo;
+            *reinterpret_cast<float4*>(sZ + (size_t)m * S + kloc) = zo;
+            *reinterpret_cast<float4*>(Ul + (size_t)m * d + k0) = uo;
+            *reinterpret_cast<float4*>(Zl + (size_t)m * d + k0) = zo;
         }
-        // ---- true pivot column of W, scaled: c = W[:,p] / sqrt(h)
-        if (tid < rp) {
-            double w = (tid < r) ? (double)Wl[(size_t)p * rp + tid] : 0.0;
-            for (int s = 0; s < m; ++s) w = fma(-(double)Cl[(size_t)s * rp + tid], (double)sUp[s], w);
-            Cl[(size_t)m * rp + tid] = (float)(w * rs);
+        // no barrier here: the next step's cluster barrier orders these writes before any read
+    }
+    cluster.sync();
+
+    // ---- c_m = (W[:,p_m] - sum_{s<m} c_s T[m][s]) / sqrt(h_m): forward substitution per row
+    //      index i of W, each CTA takes a slice of the d_row indices
+    {
+        const int per = (rp + CS - 1) / CS;
+        for (int i = rank * per + tid; i < min(rp, (rank + 1) * per); i += STEP_THREADS) {
+            float w[BMAX], c[BMAX];
+#pragma unroll
+            for (int m = 0; m < BMAX; ++m)
+                w[m] = (m < nsteps && i < r) ? Wl[(size_t)s_pm[m] * rp + i] : 0.f;
+#pragma unroll
+            for (int m = 0; m < BMAX; ++m) {
+                double acc = (double)w[m];
+#pragma unroll
+                for (int s = 0; s < m; ++s) acc = fma(-(double)c[s], (double)sT[m][s], acc);
+                c[m] = (m < nsteps) ? (float)(acc * s_rsm[m]) : 0.f;
+                if (m < nsteps) Cl[(size_t)m * rp + i] = c[m];
+            }
         }
-        __syncthreads();
     }
 
-    // ---- stable compaction of the per-position vectors; src[new] = old position
-    int base = 0;
+    // ---- stable compaction of the per-position vectors across the cluster; src[new] = old
+    const int f0 = alive[0] ? 1 : 0, f1 = alive[1] ? 1 : 0, f2 = alive[2] ? 1 : 0, f3 = alive[3] ? 1 : 0;
+    const int mine = f0 + f1 + f2 + f3;
+    int incl = mine;
 #pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const int k = tid + STEP_THREADS * j;
-        const int f = alive[j] ? 1 : 0;
-        int incl = f;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) s_scan[warp] = incl;
-        __syncthreads();
-        if (warp == 0) {
-            int w = s_scan[lane], wi = w;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, wi, o);
-                if (lane >= o) wi += v;
-            }
-            s_scan[lane] = wi - w;          // exclusive prefix of the warp totals
-            if (lane == 31) s_p = wi;       // chunk total
-        }
-        __syncthreads();
-        if (f) {
-            const int np = base + s_scan[warp] + incl - 1;
-            src[(size_t)l * d + np] = k;
-            dA_out[(size_t)l * d + np] = da[j];
-            dQ_out[(size_t)l * d + np] = dq[j];
-            idx_out[(size_t)l * d + np] = org[j];
-        }
-        base += s_p;
-        __syncthreads();
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
     }
-    if (tid == 0) state[l].n_new = base;
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    if (tid == 0) {
+        int t = 0;
+        for (int w2 = 0; w2 < NW; ++w2) { const int v = s_wsum[w2]; s_wsum[w2] = t; t += v; }
+        s_count = t;
+    }
+    cluster.sync();
+    int base = 0;
+    for (int c2 = 0; c2 < rank; ++c2) base += *cluster.map_shared_rank(&s_count, c2);
+    int np = base + s_wsum[warp] + incl - mine;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        if (alive[e]) {
+            src[(size_t)l * d + np] = k0 + e;
+            dA_out[(size_t)l * d + np] = da[e];
+            dQ_out[(size_t)l * d + np] = dq[e];
+            idx_out[(size_t)l * d + np] = org[e];
+            ++np;
+        }
+    }
+    if (rank == 0 && tid == 0) state[l].sumrho += sumrho;
+    if (rank == CS - 1 && tid == 0) state[l].n_new = base + s_count;
+    cluster.sync();      // no CTA may retire while another can still read its shared memory
 }
 
 // Rank-m update of the strict lower triangles of H^-1 and Q with compaction (out of place):
@@ -516,7 +592,7 @@ LazyWs carve_lazy(void* ws, int L, int r, int d) {
 
 }  // namespace
 
-bool lazy_path_supported(int d) { return d % 4 == 0 && d <= KPT * STEP_THREADS && d >= 4; }
+bool lazy_path_supported(int d) { return d % 4 == 0 && d <= CLUSTER_MAX * SLICE_MAX && d >= 4; }
 
 size_t lazy_workspace_bytes(int L, int r, int d, int n_levels) {
     (void)n_levels;
@@ -562,6 +638,8 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
     s = init();
     if (s != ZIPLM_OK) return s;
 
+    ZIPLM_CHECK_CUDA(cudaFuncSetAttribute(k_lazy_steps, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          2 * BMAX * SLICE_MAX * (int)sizeof(float)));
     int cur = 0;
     auto snapshot = [&](int n, int slot) -> ziplm_status {
         PhaseScope ps(PH_SNAPSHOT, st);
@@ -587,10 +665,27 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
         const int nxt = cur ^ 1;
         {
             PhaseScope ps(PH_LAZY_STEPS, st);
-            k_lazy_steps<<<L, STEP_THREADS, 0, st>>>(n, t, nsteps, d, G, r, rp, w.A[cur], w.Q[cur],
-                                                    w.Wt[cur], w.dA[cur], w.dQ[cur], w.idx[cur],
-                                                    w.dA[nxt], w.dQ[nxt], w.idx[nxt], w.src, w.U, w.Z,
-                                                    w.C, w.state, order, saliency, layer_status);
+            // smallest cluster whose per-CTA slice of positions fits shared memory
+            int cs = 1;
+            while (cs < CLUSTER_MAX && round_up_int((n + cs - 1) / cs, 4) > SLICE_MAX) cs *= 2;
+            const int S = round_up_int((n + cs - 1) / cs, 4);
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(L * cs);
+            cfg.blockDim = dim3(STEP_THREADS);
+            cfg.dynamicSmemBytes = (size_t)2 * BMAX * S * sizeof(float);
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = cs;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            ZIPLM_CHECK_CUDA(cudaLaunchKernelEx(
+                &cfg, k_lazy_steps, n, S, t, nsteps, d, G, r, rp, (const float*)w.A[cur],
+                (const float*)w.Q[cur], (const float*)w.Wt[cur], (const double*)w.dA[cur],
+                (const double*)w.dQ[cur], (const int*)w.idx[cur], w.dA[nxt], w.dQ[nxt], w.idx[nxt],
+                w.src, w.U, w.Z, w.C, w.state, order, saliency, layer_status));
             ZIPLM_CHECK_LAUNCH();
         }
         const int n_new = n - nsteps;
