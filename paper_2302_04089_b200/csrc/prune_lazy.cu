@@ -427,36 +427,59 @@ __global__ void __launch_bounds__(256) k_lazy_update_aq(int n_new, int m, int d,
 }
 
 // Rank-m update of W^T with row compaction (out of place): Wt'[i,:] = Wt[si,:] - sum_s U[s,si] C[s,:].
+// A CTA owns 64 rows x 256 columns; the C panel and the rows' U entries are staged in shared
+// memory once per CTA, each thread carries 16 rows of one float4 column.
 __global__ void __launch_bounds__(256) k_lazy_update_w(int n_new, int m, int d, int rp,
                                                        const float* __restrict__ Wt,
                                                        float* __restrict__ Wt2,
                                                        const int* __restrict__ src,
                                                        const float* __restrict__ U,
                                                        const float* __restrict__ C) {
-    const int l = blockIdx.y;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int i = blockIdx.x * 8 + warp;
-    if (i >= n_new) return;
-    const int si = src[(size_t)l * d + i];
+    __shared__ float4 sC[BMAX][64];       // C[s][col0 .. col0+255]
+    __shared__ float sUr[BMAX][64];       // U[s][src[row]]
+    __shared__ int srow[64];
+    const int l = blockIdx.z;
+    const int i0 = blockIdx.x * 64, c0 = blockIdx.y * 256;
+    const int tid = threadIdx.x, tx = tid & 63, ty = tid >> 6;      // ty: rows ty, ty+4, ...
+    if (tid < 64) srow[tid] = (i0 + tid < n_new) ? src[(size_t)l * d + i0 + tid] : -1;
+    __syncthreads();
     const float* Ul = U + (size_t)l * BMAX * d;
-    const float4* Cl = reinterpret_cast<const float4*>(C + (size_t)l * BMAX * rp);
-    const float4* in = reinterpret_cast<const float4*>(Wt + (size_t)l * d * rp + (size_t)si * rp);
-    float4* out = reinterpret_cast<float4*>(Wt2 + (size_t)l * d * rp + (size_t)i * rp);
-    float us[BMAX];
+    const float* Cl = C + (size_t)l * BMAX * rp;
+    for (int e = tid; e < m * 64; e += 256) {
+        const int s = e >> 6, c = e & 63;
+        const int sr = srow[c];
+        sUr[s][c] = sr >= 0 ? Ul[(size_t)s * d + sr] : 0.f;
+        const int col = c0 + 4 * c;
+        sC[s][c] = (col < rp) ? *reinterpret_cast<const float4*>(Cl + (size_t)s * rp + col)
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int col = c0 + 4 * tx;
+    const bool col_ok = col < rp;
+    float4 w[16];
 #pragma unroll
-    for (int s = 0; s < BMAX; ++s) us[s] = (s < m) ? Ul[(size_t)s * d + si] : 0.f;
-    const int nvec = rp >> 2;
-    for (int v = lane; v < nvec; v += 32) {
-        float4 w = __ldcs(in + v);
+    for (int x = 0; x < 16; ++x) {
+        const int sr = srow[ty + 4 * x];
+        w[x] = (sr >= 0 && col_ok)
+                   ? __ldcs(reinterpret_cast<const float4*>(Wt + (size_t)l * d * rp + (size_t)sr * rp + col))
+                   : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    __syncthreads();
+    for (int s = 0; s < m; ++s) {
+        const float4 c = sC[s][tx];
 #pragma unroll
-        for (int s = 0; s < BMAX; ++s) {
-            if (s < m) {
-                const float4 c = __ldg(Cl + (size_t)s * nvec + v);
-                w.x = fmaf(-us[s], c.x, w.x); w.y = fmaf(-us[s], c.y, w.y);
-                w.z = fmaf(-us[s], c.z, w.z); w.w = fmaf(-us[s], c.w, w.w);
-            }
+        for (int x = 0; x < 16; ++x) {
+            const float nu = -sUr[s][ty + 4 * x];
+            w[x].x = fmaf(nu, c.x, w[x].x); w[x].y = fmaf(nu, c.y, w[x].y);
+            w[x].z = fmaf(nu, c.z, w[x].z); w[x].w = fmaf(nu, c.w, w[x].w);
         }
-        out[v] = w;
+    }
+    if (col_ok) {
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+            const int i = i0 + ty + 4 * x;
+            if (i < n_new)
+                *reinterpret_cast<float4*>(Wt2 + (size_t)l * d * rp + (size_t)i * rp + col) = w[x];
+        }
     }
 }
 
@@ -700,8 +723,8 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
         }
         if (n_new > 0) {
             PhaseScope ps(PH_LAZY_UPDATE_W, st);
-            k_lazy_update_w<<<dim3((n_new + 7) / 8, L), 256, 0, st>>>(n_new, nsteps, d, rp, w.Wt[cur],
-                                                                     w.Wt[nxt], w.src, w.U, w.C);
+            k_lazy_update_w<<<dim3((n_new + 63) / 64, (rp + 255) / 256, L), 256, 0, st>>>(
+                n_new, nsteps, d, rp, w.Wt[cur], w.Wt[nxt], w.src, w.U, w.C);
             ZIPLM_CHECK_LAUNCH();
         }
         cur = nxt;
