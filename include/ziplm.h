@@ -5,11 +5,14 @@
  * Conventions shared by every entry point
  *   - "dev" pointers are CUDA device pointers of the current device, "host" pointers are
  *     ordinary host memory.  All matrices are dense row-major.
- *   - The caller owns every buffer.  The library allocates no device memory, creates no stream
- *     and keeps no state between calls (the optional diagnostics at the end of this file aside).
- *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = the default
- *     stream) and the call returns without synchronising.  Buffers must stay alive until the
- *     stream has drained.
+ *   - The caller owns every buffer.  The library allocates no device memory and keeps no state
+ *     between calls (the optional diagnostics at the end of this file aside).
+ *   - All work is ordered on `cuda_stream` (a cudaStream_t passed as void*, NULL = the default
+ *     stream) and the call returns without synchronising: it starts after everything already
+ *     enqueued there and the stream continues only when it is complete.  Buffers must stay alive
+ *     until the stream has drained.  ziplm_prune_layers may run groups of layers concurrently on
+ *     up to four internal non-blocking streams (created once per device, on first use), forked
+ *     from and joined back to `cuda_stream` with events.
  *   - The return value reports what the host can see when the work is enqueued (bad arguments,
  *     workspace too small, a failed launch).  Failures that depend on the data (a Hessian that
  *     is not positive definite, non-finite values) are written to `layer_status[l]` on the
@@ -105,16 +108,16 @@ ziplm_status ziplm_damped_inverse(const float* H, int L, int d, float damp_frac,
  * process whose whole device budget was handed to another allocator up front, or a real-time
  * loop where a cudaMalloc (which may synchronise the device) is not acceptable.  For them this
  * entry point computes exactly what ziplm_damped_inverse computes, with the same kernels, but
- * takes its scratch from an 8 MiB array that is compiled into the library.  It calls neither
+ * takes its scratch from a 12 MiB array that is compiled into the library.  It calls neither
  * cudaMalloc nor cudaFree nor any routine that allocates.
  *
  *   H, Hinv, layer_status, damp_frac, cuda_stream   as for ziplm_damped_inverse; the caller still
  *                 provides the input and both outputs.
  *
- * Limit: the request must satisfy ziplm_inverse_workspace_bytes(L, d) <= 8 MiB (8388608), e.g.
+ * Limit: the request must satisfy ziplm_inverse_workspace_bytes(L, d) <= 12 MiB (12582912), e.g.
  * one layer up to d = 704, four layers of d = 320, sixteen layers of d = 128; anything larger
  * returns ZIPLM_ERR_UNSUPPORTED and does nothing.
- * Cost: every GPU that loads the library holds the 8 MiB until the process exits.
+ * Cost: every GPU that loads the library holds the 12 MiB until the process exits.
  * First call on a device: it looks up the device address of the built-in array (with that
  * device current) and remembers it; make this first call outside any stream capture.
  * Sharing: all calls on a device use the same array, and it keeps whatever the last call left

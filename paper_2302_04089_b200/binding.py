@@ -174,9 +174,9 @@ def damped_inverse_noalloc(H: torch.Tensor, damp_frac: float, Hinv: torch.Tensor
                            layer_status: torch.Tensor) -> None:
     """ziplm_damped_inverse_noalloc: the damped inverse for callers that must not allocate.
 
-    The scratch comes from an 8 MiB array inside the library, so this wrapper allocates nothing
+    The scratch comes from a 12 MiB array inside the library, so this wrapper allocates nothing
     either: the caller passes the input H [L, d, d] fp32 and both outputs, Hinv [L, d, d]
-    float64 and layer_status [L] int32.  Requests with inverse_workspace_bytes(L, d) > 8 MiB
+    float64 and layer_status [L] int32.  Requests with inverse_workspace_bytes(L, d) > 12 MiB
     raise ZiplmError(ERR_UNSUPPORTED).  Calls that overlap on the GPU race on the shared scratch.
     """
     lib = load_library()

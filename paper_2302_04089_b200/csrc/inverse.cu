@@ -1,10 +1,14 @@
 // Damped float64 inverse of the calibration Hessian (caption of Algorithm 1:
 // H^-1 = (2 X X^T + lambda I)^-1), batched over layers.
 //
-// Route: H + lambda I = C C^T by a left-looking blocked Cholesky (64 x 64 tiles), M = C^-1 by
-// block forward substitution along tile anti-diagonals, H^-1 = M^T M.  Everything is float64:
-// the greedy loop that follows needs the diagonal of H^-1 to roughly 1e-7 relative, which an
-// fp32 factorisation of a matrix with condition number 1e3 .. 1e5 does not give.  The matrix is
+// Route: H + lambda I = F F^T (Cholesky), M = F^-1, H^-1 = M^T M, all on 64 x 64 tiles.  The
+// factor and its inverse are built together by recursive halving of the tile range [lo, hi):
+//     factor [lo, mid);   F21 = A21 M11^T;   A22 -= F21 F21^T;   factor [mid, hi);
+//     M21 = -M22 (F21 M11)
+// so that nearly all of the work sits in large, wide products (thousands of independent tiles
+// per launch) and only the 64 x 64 leaves are sequential.  Everything is float64: the greedy
+// loop that follows needs the diagonal of H^-1 to roughly 1e-7 relative, which an fp32
+// factorisation of a matrix with condition number 1e3 .. 1e5 does not give.  The matrix is
 // padded to a multiple of 64 with an identity block, whose inverse is again the identity.
 #include <math.h>
 
@@ -15,72 +19,96 @@
 // Built-in scratch of ziplm_damped_inverse_noalloc: lives in every GPU that loads this library
 // until the process exits.  In host code this name is only a handle for cudaGetSymbolAddress,
 // never a device address.
-constexpr size_t kBuiltinScratchBytes = (size_t)8 << 20;
+constexpr size_t kBuiltinScratchBytes = (size_t)12 << 20;
 static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
 
 namespace ziplm {
 namespace {
-
 constexpr int KC = 16;          // k-chunk staged in shared memory per iteration
 constexpr int LDS = kTile + 2;  // padded shared-memory row length (doubles)
+constexpr int GT = 128;         // threads of a product CTA: 8 x 4 outputs per thread
 
-// acc(64x64) += opA(64xK) * opB(Kx64); 256 threads, thread (ty,tx) owns rows ty+16a, cols tx+16b.
-//   TA == false: A stored 64 x K row-major (opA(i,k) = A[i*lda + k]); true: stored K x 64.
-//   TB == false: B stored K x 64 row-major (opB(k,j) = B[k*ldb + j]); true: stored 64 x K.
-// Ends with __syncthreads(), so the caller may overwrite the operands afterwards.  The operand
-// pointers are deliberately not __restrict__: some callers read tiles that the same block wrote
-// earlier in the kernel, which must not go through the non-coherent load path.
-template <bool TA, bool TB>
-__device__ __forceinline__ void dgemm_tile(double (&acc)[4][4], const double* A, int lda,
-                                           const double* B, int ldb, int K,
-                                           double (*sA)[LDS], double (*sB)[LDS]) {
+struct TileSmem {
+    double a[2][KC][LDS];
+    double b[2][KC][LDS];
+};
+
+// Fetch one 64 x KC chunk of an operand into registers (8 doubles per thread).
+//   T == false: stored 64 x K row-major (op(i,k) = P[i*ld + k]); true: stored K x 64.
+template <bool T>
+__device__ __forceinline__ void chunk_load(double (&r)[8], const double* P, int ld, int k0) {
     const int tid = threadIdx.x;
-    const int ty = tid >> 4, tx = tid & 15;
-    for (int k0 = 0; k0 < K; k0 += KC) {
-        if (!TA) {
-            const int i = tid >> 2, kq = (tid & 3) * 4;
-            const double* src = A + (size_t)i * lda + k0 + kq;
-            const double2 v0 = *reinterpret_cast<const double2*>(src);
-            const double2 v1 = *reinterpret_cast<const double2*>(src + 2);
-            sA[kq][i] = v0.x; sA[kq + 1][i] = v0.y; sA[kq + 2][i] = v1.x; sA[kq + 3][i] = v1.y;
-        } else {
-            const int kk = tid >> 4, iq = (tid & 15) * 4;
-            const double* src = A + (size_t)(k0 + kk) * lda + iq;
-            const double2 v0 = *reinterpret_cast<const double2*>(src);
-            const double2 v1 = *reinterpret_cast<const double2*>(src + 2);
-            sA[kk][iq] = v0.x; sA[kk][iq + 1] = v0.y; sA[kk][iq + 2] = v1.x; sA[kk][iq + 3] = v1.y;
-        }
-        if (!TB) {
-            const int kk = tid >> 4, jq = (tid & 15) * 4;
-            const double* src = B + (size_t)(k0 + kk) * ldb + jq;
-            const double2 v0 = *reinterpret_cast<const double2*>(src);
-            const double2 v1 = *reinterpret_cast<const double2*>(src + 2);
-            sB[kk][jq] = v0.x; sB[kk][jq + 1] = v0.y; sB[kk][jq + 2] = v1.x; sB[kk][jq + 3] = v1.y;
-        } else {
-            const int j = tid >> 2, kq = (tid & 3) * 4;
-            const double* src = B + (size_t)j * ldb + k0 + kq;
-            const double2 v0 = *reinterpret_cast<const double2*>(src);
-            const double2 v1 = *reinterpret_cast<const double2*>(src + 2);
-            sB[kq][j] = v0.x; sB[kq + 1][j] = v0.y; sB[kq + 2][j] = v1.x; sB[kq + 3][j] = v1.y;
-        }
-        __syncthreads();
+    const double* src = T ? P + (size_t)(k0 + (tid >> 3)) * ld + (tid & 7) * 8
+                          : P + (size_t)(tid >> 1) * ld + k0 + (tid & 1) * 8;
 #pragma unroll
-        for (int kk = 0; kk < KC; ++kk) {
-            double a[4], b[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) { a[q] = sA[kk][ty + 16 * q]; b[q] = sB[kk][tx + 16 * q]; }
-#pragma unroll
-            for (int p = 0; p < 4; ++p)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) acc[p][q] = fma(a[p], b[q], acc[p][q]);
-        }
-        __syncthreads();
+    for (int e = 0; e < 4; ++e) {
+        const double2 v = *reinterpret_cast<const double2*>(src + 2 * e);
+        r[2 * e] = v.x; r[2 * e + 1] = v.y;
     }
 }
 
-__device__ __forceinline__ void zero_acc(double (&acc)[4][4]) {
+template <bool T>
+__device__ __forceinline__ void chunk_store(double (*s)[LDS], const double (&r)[8]) {
+    const int tid = threadIdx.x;
+    if (T) {
+        const int kk = tid >> 3, iq = (tid & 7) * 8;
 #pragma unroll
-    for (int p = 0; p < 4; ++p)
+        for (int e = 0; e < 8; ++e) s[kk][iq + e] = r[e];
+    } else {
+        const int i = tid >> 1, kq = (tid & 1) * 8;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) s[kq + e][i] = r[e];
+    }
+}
+
+// acc(64x64) += opA(64xK) * opB(Kx64); 128 threads, thread (ty,tx) owns rows ty+8a (a < 8) and
+// cols tx+16b (b < 4).  The next chunk is fetched into registers while the current one is
+// multiplied out of shared memory (two buffers, one barrier per chunk).  The operand pointers
+// are deliberately not __restrict__: callers may read tiles written earlier in the same launch
+// sequence.  Ends with __syncthreads().
+template <bool TA, bool TB>
+__device__ __forceinline__ void dgemm_tile(double (&acc)[8][4], const double* A, int lda,
+                                           const double* B, int ldb, int K, TileSmem& sm) {
+    const int tid = threadIdx.x;
+    const int ty = tid >> 4, tx = tid & 15;
+    if (K <= 0) return;
+    double ra[8], rb[8];
+    chunk_load<TA>(ra, A, lda, 0);
+    chunk_load<TB ? false : true>(rb, B, ldb, 0);
+    chunk_store<TA>(sm.a[0], ra);
+    chunk_store<TB ? false : true>(sm.b[0], rb);
+    __syncthreads();
+    int buf = 0;
+    for (int k0 = 0; k0 < K; k0 += KC) {
+        const bool more = k0 + KC < K;
+        if (more) {
+            chunk_load<TA>(ra, A, lda, k0 + KC);
+            chunk_load<TB ? false : true>(rb, B, ldb, k0 + KC);
+        }
+#pragma unroll
+        for (int kk = 0; kk < KC; ++kk) {
+            double a[8], b[4];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) a[q] = sm.a[buf][kk][ty + 8 * q];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) b[q] = sm.b[buf][kk][tx + 16 * q];
+#pragma unroll
+            for (int p = 0; p < 8; ++p)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[p][q] = fma(a[p], b[q], acc[p][q]);
+        }
+        if (more) {
+            chunk_store<TA>(sm.a[buf ^ 1], ra);
+            chunk_store<TB ? false : true>(sm.b[buf ^ 1], rb);
+        }
+        __syncthreads();
+        buf ^= 1;
+    }
+}
+
+__device__ __forceinline__ void zero_acc(double (&acc)[8][4]) {
+#pragma unroll
+    for (int p = 0; p < 8; ++p)
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[p][q] = 0.0;
 }
@@ -152,36 +180,68 @@ __global__ void __launch_bounds__(256) k_fill_damped(const float* __restrict__ H
     if (bad) set_layer_status(layer_status, l, ZIPLM_ERR_NONFINITE);
 }
 
-// Left-looking update of block column j: C_ij -= sum_{k<j} C_ik C_jk^T for tiles i >= j.
-__global__ void __launch_bounds__(256) k_chol_update(double* C, int dp, int j) {
-    __shared__ double sA[KC][LDS], sB[KC][LDS];
+// One launch of the recursion: C_out[tile (ti,tj)] = beta * C_out + alpha * sum_k opA(ti,k) opB(k,tj)
+// over a rectangle of mt x nt tiles, with the k range cut to the non-zero tiles of a triangular
+// operand.  All matrices are dp x dp float64 per layer; coordinates are in tiles.
+struct GemmTask {
+    const double* A; int a_r, a_c;      // TA == false: tile (ti,k) at (a_r + ti, a_c + k); true: (a_r + k, a_c + ti)
+    const double* B; int b_r, b_c;      // TB == false: tile (k,tj) at (b_r + k, b_c + tj); true: (b_r + tj, b_c + k)
+    double* C; int c_r, c_c;
+    int mt, nt, kt;
+    int kmode;                          // 0: all k; 1: k <= tj; 2: k <= ti; 3: k >= tj
+    int lower_only;                     // square region: only tiles ti >= tj
+    double alpha; int beta;             // beta in {0, 1}
+};
+
+template <bool TA, bool TB>
+__global__ void __launch_bounds__(GT) k_dgemm_tiles(GemmTask t, int dp) {
+    __shared__ TileSmem sm;
     const int l = blockIdx.y;
-    const int i = j + blockIdx.x;
-    double* Cl = C + (size_t)l * dp * dp;
-    double acc[4][4];
+    int ti, tj;
+    if (t.lower_only) {
+        ti = 0; int rem = blockIdx.x;
+        while (rem > ti) { rem -= ti + 1; ++ti; }
+        tj = rem;
+    } else {
+        ti = blockIdx.x / t.nt; tj = blockIdx.x % t.nt;
+    }
+    int klo = 0, khi = t.kt;
+    if (t.kmode == 1) khi = min(t.kt, tj + 1);
+    else if (t.kmode == 2) khi = min(t.kt, ti + 1);
+    else if (t.kmode == 3) klo = tj;
+    const size_t lay = (size_t)l * dp * dp;
+    const double* A = t.A + lay + (TA ? ((size_t)(t.a_r + klo) * kTile * dp + (size_t)(t.a_c + ti) * kTile)
+                                      : ((size_t)(t.a_r + ti) * kTile * dp + (size_t)(t.a_c + klo) * kTile));
+    const double* B = t.B + lay + (TB ? ((size_t)(t.b_r + tj) * kTile * dp + (size_t)(t.b_c + klo) * kTile)
+                                      : ((size_t)(t.b_r + klo) * kTile * dp + (size_t)(t.b_c + tj) * kTile));
+    double acc[8][4];
     zero_acc(acc);
-    dgemm_tile<false, true>(acc, Cl + (size_t)i * kTile * dp, dp, Cl + (size_t)j * kTile * dp, dp,
-                            j * kTile, sA, sB);
+    dgemm_tile<TA, TB>(acc, A, dp, B, dp, (khi - klo) * kTile, sm);
+    double* out = t.C + lay + (size_t)(t.c_r + ti) * kTile * dp + (size_t)(t.c_c + tj) * kTile;
     const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
-    double* out = Cl + (size_t)i * kTile * dp + (size_t)j * kTile;
 #pragma unroll
-    for (int p = 0; p < 4; ++p)
+    for (int p = 0; p < 8; ++p)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) out[(size_t)(ty + 16 * p) * dp + tx + 16 * q] -= acc[p][q];
+        for (int q = 0; q < 4; ++q) {
+            double* o = out + (size_t)(ty + 8 * p) * dp + tx + 16 * q;
+            const double v = t.alpha * acc[p][q];
+            *o = t.beta ? (*o + v) : v;
+        }
 }
 
-// Unblocked Cholesky of the diagonal tile C_jj (in place, lower) and the inverse of its factor.
-__global__ void __launch_bounds__(256) k_potf2(double* C, int dp, int T, int j, double* Linv,
+// Leaf of the recursion: unblocked Cholesky of the diagonal tile A_jj -> F_jj (lower, upper part
+// zeroed) and the inverse of that factor -> M_jj (lower, upper part zeroed).
+__global__ void __launch_bounds__(256) k_potf2(const double* A, double* F, double* M, int dp, int j,
                                                int* layer_status) {
     __shared__ double s[kTile][kTile + 1];
-    __shared__ double dinv[kTile];   // diagonal of the inverse factor
+    __shared__ double dinv[kTile];
     __shared__ int sflag;
     const int l = blockIdx.x;
-    const int tid = threadIdx.x;
-    double* tile = C + (size_t)l * dp * dp + (size_t)j * kTile * dp + (size_t)j * kTile;
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const size_t off = (size_t)l * dp * dp + (size_t)j * kTile * dp + (size_t)j * kTile;
     if (tid == 0) sflag = 0;
     for (int e = tid; e < kTile * kTile; e += 256)
-        s[e >> 6][e & 63] = tile[(size_t)(e >> 6) * dp + (e & 63)];
+        s[e >> 6][e & 63] = A[off + (size_t)(e >> 6) * dp + (e & 63)];
     __syncthreads();
     for (int c = 0; c < kTile; ++c) {
         if (tid == 0) {
@@ -195,11 +255,17 @@ __global__ void __launch_bounds__(256) k_potf2(double* C, int dp, int T, int j, 
         __syncthreads();
         if (tid > c && tid < kTile) s[tid][c] /= s[c][c];
         __syncthreads();
-        // trailing update of the lower triangle: (i, jj) with c < jj <= i < 64
-        const int m = kTile - 1 - c;
-        for (int e = tid; e < m * m; e += 256) {
-            const int i = c + 1 + e / m, jj = c + 1 + e % m;
-            if (jj <= i) s[i][jj] -= s[i][c] * s[jj][c];
+        // trailing update of the lower triangle: rows ty + 16a, cols tx + 16b
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const int i = ty + 16 * a;
+            if (i <= c) continue;
+            const double lic = s[i][c];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int jj = tx + 16 * b;
+                if (jj > c && jj <= i) s[i][jj] -= lic * s[jj][c];
+            }
         }
         __syncthreads();
     }
@@ -210,100 +276,48 @@ __global__ void __launch_bounds__(256) k_potf2(double* C, int dp, int T, int j, 
         const int cidx = tid;
         dinv[cidx] = 1.0 / s[cidx][cidx];
         for (int i = cidx + 1; i < kTile; ++i) {
-            double acc = -s[i][cidx] * dinv[cidx];
-            for (int k = cidx + 1; k < i; ++k) acc -= s[i][k] * s[cidx][k];
-            s[cidx][i] = acc / s[i][i];
+            double a0 = -s[i][cidx] * dinv[cidx], a1 = 0.0, a2 = 0.0, a3 = 0.0;
+            int k = cidx + 1;
+            for (; k + 3 < i; k += 4) {
+                a0 = fma(-s[i][k], s[cidx][k], a0);
+                a1 = fma(-s[i][k + 1], s[cidx][k + 1], a1);
+                a2 = fma(-s[i][k + 2], s[cidx][k + 2], a2);
+                a3 = fma(-s[i][k + 3], s[cidx][k + 3], a3);
+            }
+            for (; k < i; ++k) a0 = fma(-s[i][k], s[cidx][k], a0);
+            s[cidx][i] = ((a0 + a1) + (a2 + a3)) / s[i][i];
         }
     }
     __syncthreads();
-    double* li = Linv + ((size_t)l * T + j) * kTile * kTile;
     for (int e = tid; e < kTile * kTile; e += 256) {
         const int i = e >> 6, jj = e & 63;
-        tile[(size_t)i * dp + jj] = (jj <= i) ? s[i][jj] : 0.0;
-        li[e] = (jj < i) ? s[jj][i] : (jj == i ? dinv[i] : 0.0);
+        F[off + (size_t)i * dp + jj] = (jj <= i) ? s[i][jj] : 0.0;
+        M[off + (size_t)i * dp + jj] = (jj < i) ? s[jj][i] : (jj == i ? dinv[i] : 0.0);
     }
     if (tid == 0 && sflag) set_layer_status(layer_status, l, sflag);
 }
 
-// Panel below the diagonal tile: C_ij <- C_ij * inv(C_jj)^T for i > j.
-__global__ void __launch_bounds__(256) k_chol_panel(double* C, int dp, int T, int j,
-                                                    const double* Linv) {
-    __shared__ double sA[KC][LDS], sB[KC][LDS];
-    const int l = blockIdx.y;
-    const int i = j + 1 + blockIdx.x;
-    double* tile = C + (size_t)l * dp * dp + (size_t)i * kTile * dp + (size_t)j * kTile;
-    const double* li = Linv + ((size_t)l * T + j) * kTile * kTile;
-    double acc[4][4];
-    zero_acc(acc);
-    dgemm_tile<false, true>(acc, tile, dp, li, kTile, kTile, sA, sB);
-    const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
-#pragma unroll
-    for (int p = 0; p < 4; ++p)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) tile[(size_t)(ty + 16 * p) * dp + tx + 16 * q] = acc[p][q];
-}
-
-// M_jj = inv(C_jj) for every diagonal tile.
-__global__ void __launch_bounds__(256) k_trtri_diag(double* M, int dp, int T, const double* Linv) {
-    const int l = blockIdx.y, j = blockIdx.x;
-    double* tile = M + (size_t)l * dp * dp + (size_t)j * kTile * dp + (size_t)j * kTile;
-    const double* li = Linv + ((size_t)l * T + j) * kTile * kTile;
-    for (int e = threadIdx.x; e < kTile * kTile; e += 256)
-        tile[(size_t)(e >> 6) * dp + (e & 63)] = li[e];
-}
-
-// Tiles on anti-diagonal s of M = C^-1:  M_ij = -inv(C_ii) * sum_{k=j}^{i-1} C_ik M_kj, i = j + s.
-__global__ void __launch_bounds__(256) k_trtri_offdiag(const double* C, double* M, int dp, int T,
-                                                       int s, const double* Linv) {
-    __shared__ double sA[KC][LDS], sB[KC][LDS];
-    const int l = blockIdx.y;
-    const int j = blockIdx.x, i = j + s;
-    const double* Cl = C + (size_t)l * dp * dp;
-    double* Ml = M + (size_t)l * dp * dp;
-    double* tile = Ml + (size_t)i * kTile * dp + (size_t)j * kTile;
-    const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
-    double acc[4][4];
-    zero_acc(acc);
-    dgemm_tile<false, false>(acc, Cl + (size_t)i * kTile * dp + (size_t)j * kTile, dp,
-                             Ml + (size_t)j * kTile * dp + (size_t)j * kTile, dp, s * kTile, sA, sB);
-    // park the partial sum in the output tile (this block owns it), then multiply by -inv(C_ii)
-#pragma unroll
-    for (int p = 0; p < 4; ++p)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) tile[(size_t)(ty + 16 * p) * dp + tx + 16 * q] = acc[p][q];
-    __syncthreads();
-    zero_acc(acc);
-    dgemm_tile<false, false>(acc, Linv + ((size_t)l * T + i) * kTile * kTile, kTile, tile, dp, kTile,
-                             sA, sB);
-#pragma unroll
-    for (int p = 0; p < 4; ++p)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) tile[(size_t)(ty + 16 * p) * dp + tx + 16 * q] = -acc[p][q];
-}
-
 // H^-1 = M^T M on the lower tiles (i >= j): sum over k >= i of M_ki^T M_kj; writes the cropped
 // d x d result as float64 (mirrored to the upper triangle) and/or fp32 strict lower + fp64 diag.
-__global__ void __launch_bounds__(256) k_lauum(const double* M, int dp, int T, int d,
-                                               double* out64, float* tri32, int pitch32,
-                                               double* diag64) {
-    __shared__ double sA[KC][LDS], sB[KC][LDS];
+__global__ void __launch_bounds__(GT) k_lauum(const double* M, int dp, int T, int d, double* out64,
+                                              float* tri32, int pitch32, double* diag64) {
+    __shared__ TileSmem sm;
     const int l = blockIdx.y;
     // linear tile index -> (i, j), rows of the lower triangle in order i = 0, 1, ...
     int i = 0, rem = blockIdx.x;
     while (rem > i) { rem -= i + 1; ++i; }
     const int j = rem;
     const double* Ml = M + (size_t)l * dp * dp;
-    double acc[4][4];
+    double acc[8][4];
     zero_acc(acc);
     dgemm_tile<true, false>(acc, Ml + (size_t)i * kTile * dp + (size_t)i * kTile, dp,
-                            Ml + (size_t)i * kTile * dp + (size_t)j * kTile, dp, (T - i) * kTile, sA,
-                            sB);
+                            Ml + (size_t)i * kTile * dp + (size_t)j * kTile, dp, (T - i) * kTile, sm);
     const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
 #pragma unroll
-    for (int p = 0; p < 4; ++p)
+    for (int p = 0; p < 8; ++p)
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const int row = i * kTile + ty + 16 * p, col = j * kTile + tx + 16 * q;
+            const int row = i * kTile + ty + 8 * p, col = j * kTile + tx + 16 * q;
             if (row >= d || col >= d) continue;
             const double v = acc[p][q];
             if (out64 && row >= col) {
@@ -317,14 +331,60 @@ __global__ void __launch_bounds__(256) k_lauum(const double* M, int dp, int T, i
         }
 }
 
+struct InvCtx {
+    double* A;   // damped Hessian, updated in place (Schur complements); dead blocks serve as scratch
+    double* F;   // Cholesky factor
+    double* M;   // inverse of the factor
+    int dp, L;
+    int* layer_status;
+    cudaStream_t st;
+};
+
+template <bool TA, bool TB>
+ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
+    const int tiles = t.lower_only ? t.mt * (t.mt + 1) / 2 : t.mt * t.nt;
+    if (tiles <= 0 || t.kt <= 0) return ZIPLM_OK;
+    k_dgemm_tiles<TA, TB><<<dim3(tiles, c.L), GT, 0, c.st>>>(t, c.dp);
+    ZIPLM_CHECK_LAUNCH();
+    return ZIPLM_OK;
+}
+
+// Factor the tile range [lo, hi): on return F holds the Cholesky factor of the (updated) block
+// and M its inverse.
+ziplm_status factor_range(const InvCtx& c, int lo, int hi) {
+    if (hi - lo == 1) {
+        k_potf2<<<c.L, 256, 0, c.st>>>(c.A, c.F, c.M, c.dp, lo, c.layer_status);
+        ZIPLM_CHECK_LAUNCH();
+        return ZIPLM_OK;
+    }
+    const int mid = lo + (hi - lo) / 2;
+    const int n1 = mid - lo, n2 = hi - mid;
+    ziplm_status s = factor_range(c, lo, mid);
+    if (s != ZIPLM_OK) return s;
+    GemmTask t;
+    // F21 = A21 M11^T   (M11 lower triangular: opB(k,j) = M11[j,k] vanishes for k > j)
+    t = GemmTask{c.A, mid, lo, c.M, lo, lo, c.F, mid, lo, n2, n1, n1, 1, 0, 1.0, 0};
+    if ((s = launch_gemm<false, true>(c, t)) != ZIPLM_OK) return s;
+    // A22 -= F21 F21^T  (lower tiles)
+    t = GemmTask{c.F, mid, lo, c.F, mid, lo, c.A, mid, mid, n2, n2, n1, 0, 1, -1.0, 1};
+    if ((s = launch_gemm<false, true>(c, t)) != ZIPLM_OK) return s;
+    if ((s = factor_range(c, mid, hi)) != ZIPLM_OK) return s;
+    // scratch (the dead A21 block) = F21 M11   (M11 lower: opB(k,j) vanishes for k < j)
+    t = GemmTask{c.F, mid, lo, c.M, lo, lo, c.A, mid, lo, n2, n1, n1, 3, 0, 1.0, 0};
+    if ((s = launch_gemm<false, false>(c, t)) != ZIPLM_OK) return s;
+    // M21 = -M22 scratch  (M22 lower: opA(i,k) vanishes for k > i)
+    t = GemmTask{c.M, mid, mid, c.A, mid, lo, c.M, mid, lo, n2, n1, n2, 2, 0, -1.0, 0};
+    return launch_gemm<false, false>(c, t);
+}
+
 }  // namespace
 
 size_t inverse_workspace_bytes(int L, int d) {
-    const int dp = round_up_int(d, kTile), T = dp / kTile;
+    const int dp = round_up_int(d, kTile);
     Carver c(nullptr);
-    c.take<double>((size_t)L * dp * dp);               // C: damped Hessian -> Cholesky factor
+    c.take<double>((size_t)L * dp * dp);               // A: damped Hessian / Schur complements
+    c.take<double>((size_t)L * dp * dp);               // F: Cholesky factor
     c.take<double>((size_t)L * dp * dp);               // M: inverse of the factor
-    c.take<double>((size_t)L * T * kTile * kTile);     // inverses of the diagonal tiles
     c.take<double>((size_t)L);                         // lambda
     return c.off;
 }
@@ -335,34 +395,20 @@ ziplm_status run_damped_inverse(const float* H, int L, int d, float damp_frac, d
     if (ws_bytes < inverse_workspace_bytes(L, d)) return ZIPLM_ERR_WORKSPACE;
     const int dp = round_up_int(d, kTile), T = dp / kTile;
     Carver c(ws);
-    double* C = c.take<double>((size_t)L * dp * dp);
-    double* M = c.take<double>((size_t)L * dp * dp);
-    double* Linv = c.take<double>((size_t)L * T * kTile * kTile);
+    InvCtx ctx;
+    ctx.A = c.take<double>((size_t)L * dp * dp);
+    ctx.F = c.take<double>((size_t)L * dp * dp);
+    ctx.M = c.take<double>((size_t)L * dp * dp);
     double* lam = c.take<double>((size_t)L);
+    ctx.dp = dp; ctx.L = L; ctx.layer_status = layer_status; ctx.st = st;
 
     k_mean_diag<<<L, 256, 0, st>>>(H, d, damp_frac, lam, layer_status);
     ZIPLM_CHECK_LAUNCH();
-    k_fill_damped<<<dim3(T, dp / 16, L), 256, 0, st>>>(H, d, dp, lam, C, layer_status);
+    k_fill_damped<<<dim3(T, dp / 16, L), 256, 0, st>>>(H, d, dp, lam, ctx.A, layer_status);
     ZIPLM_CHECK_LAUNCH();
-    for (int j = 0; j < T; ++j) {
-        if (j > 0) {
-            k_chol_update<<<dim3(T - j, L), 256, 0, st>>>(C, dp, j);
-            ZIPLM_CHECK_LAUNCH();
-        }
-        k_potf2<<<L, 256, 0, st>>>(C, dp, T, j, Linv, layer_status);
-        ZIPLM_CHECK_LAUNCH();
-        if (j + 1 < T) {
-            k_chol_panel<<<dim3(T - j - 1, L), 256, 0, st>>>(C, dp, T, j, Linv);
-            ZIPLM_CHECK_LAUNCH();
-        }
-    }
-    k_trtri_diag<<<dim3(T, L), 256, 0, st>>>(M, dp, T, Linv);
-    ZIPLM_CHECK_LAUNCH();
-    for (int s = 1; s < T; ++s) {
-        k_trtri_offdiag<<<dim3(T - s, L), 256, 0, st>>>(C, M, dp, T, s, Linv);
-        ZIPLM_CHECK_LAUNCH();
-    }
-    k_lauum<<<dim3(T * (T + 1) / 2, L), 256, 0, st>>>(M, dp, T, d, out64, tri32, pitch32, diag64);
+    ziplm_status s = factor_range(ctx, 0, T);
+    if (s != ZIPLM_OK) return s;
+    k_lauum<<<dim3(T * (T + 1) / 2, L), GT, 0, st>>>(ctx.M, dp, T, d, out64, tri32, pitch32, diag64);
     ZIPLM_CHECK_LAUNCH();
     if (lam_out) {
         ZIPLM_CHECK_CUDA(cudaMemcpyAsync(lam_out, lam, sizeof(double) * L, cudaMemcpyDeviceToDevice, st));

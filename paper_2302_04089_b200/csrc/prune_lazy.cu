@@ -91,18 +91,29 @@ __global__ void __launch_bounds__(256) k_lazy_init(const float* __restrict__ W, 
     }
 }
 
+// Candidate of the argmin of rho = q / a (q = Q[k,k], a = H^-1[k,k]).  Candidates are compared by
+// cross-multiplication (q_x a_y < q_y a_x), which needs no float64 division on the critical path;
+// the quotient is formed once, for the winner.  An entry whose a is not positive or whose values
+// are not finite sorts first, so that it is picked -- and its layer flagged -- at once.
 struct Cand {
-    double rho, a, q;
+    double a, q;
     int org, pos;
 };
 
+__device__ __forceinline__ bool cand_valid(const Cand& x) {
+    return x.a > 0.0 && isfinite(x.a) && isfinite(x.q);
+}
+
 __device__ __forceinline__ bool better(const Cand& x, const Cand& y) {   // x strictly before y
-    return x.rho < y.rho || (x.rho == y.rho && x.org < y.org);
+    const bool vx = cand_valid(x), vy = cand_valid(y);
+    if (vx != vy) return !vx;
+    if (!vx) return x.org < y.org;
+    const double lhs = x.q * y.a, rhs = y.q * x.a;
+    return lhs < rhs || (lhs == rhs && x.org < y.org);
 }
 
 __device__ __forceinline__ Cand shfl_cand(const Cand& c, int off) {
     Cand o;
-    o.rho = __shfl_xor_sync(0xffffffffu, c.rho, off);
     o.a = __shfl_xor_sync(0xffffffffu, c.a, off);
     o.q = __shfl_xor_sync(0xffffffffu, c.q, off);
     o.org = __shfl_xor_sync(0xffffffffu, c.org, off);
@@ -182,13 +193,11 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
         const int par = m & 1;
         // ---- per-warp best of rho = Q[k,k] / H^-1[k,k] (ties: lowest original index)
         Cand best;
-        best.rho = INFINITY; best.a = 1.0; best.q = 0.0; best.org = 0x7fffffff; best.pos = -1;
+        best.a = 1.0; best.q = 0.0; best.org = 0x7fffffff; best.pos = -1;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (!alive[e]) continue;
             Cand c;
-            c.rho = dq[e] / da[e];
-            if (!(c.rho == c.rho)) c.rho = INFINITY;
             c.a = da[e]; c.q = dq[e]; c.org = org[e]; c.pos = k0 + e;
             merge_cand(best, c);
         }
@@ -200,7 +209,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
         //      vectors' entries at the pivot (from the CTA that owns it)
         if (warp == 0) {
             Cand g;
-            g.rho = INFINITY; g.a = 1.0; g.q = 0.0; g.org = 0x7fffffff; g.pos = -1;
+            g.a = 1.0; g.q = 0.0; g.org = 0x7fffffff; g.pos = -1;
             for (int e = lane; e < CS * NW; e += 32) {
                 const Cand* remote = cluster.map_shared_rank(&s_cand[par][e % NW], e / NW);
                 merge_cand(g, *remote);
@@ -211,7 +220,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
             if (p < 0) p = 0;
             double h = g.a;
             int bad = 0;
-            if (!isfinite(g.rho) || !isfinite(h)) { bad = ZIPLM_ERR_NONFINITE; h = 1.0; }
+            if (!isfinite(g.q) || !isfinite(h)) { bad = ZIPLM_ERR_NONFINITE; h = 1.0; }
             else if (!(h > 0.0)) { bad = ZIPLM_ERR_NOT_PD; h = 1.0; }
             const double rs = 1.0 / sqrt(h);
             const int prow = p / S, pl = p - prow * S;
@@ -230,10 +239,11 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
                 s_pm[m] = p;
                 s_rsm[m] = rs;
                 if (rank == 0) {
+                    const double rho = bad ? 0.0 : g.q / h;
                     if (bad) set_layer_status(layer_status, l, bad);
-                    sumrho += isfinite(g.rho) ? g.rho : 0.0;
+                    sumrho += rho;
                     order[(size_t)l * G + t0 + m] = g.org;
-                    if (saliency) saliency[(size_t)l * G + t0 + m] = (float)g.rho;
+                    if (saliency) saliency[(size_t)l * G + t0 + m] = (float)rho;
                 }
             }
         }
@@ -253,6 +263,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
                     q[e] = (double)Ql[off];
                 }
             }
+#pragma unroll 4
             for (int s = 0; s < m; ++s) {
                 const float4 u4 = *reinterpret_cast<const float4*>(sU + (size_t)s * S + kloc);
                 const float4 z4 = *reinterpret_cast<const float4*>(sZ + (size_t)s * S + kloc);

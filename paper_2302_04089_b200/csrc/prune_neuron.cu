@@ -384,10 +384,97 @@ static bool use_lazy_path(int d) {
     return lazy_path_supported(d);
 }
 
+// The delayed-update variant has latency-bound phases (the per-step cluster kernel occupies a
+// few dozen SMs, the panel steps of the factorisation even fewer).  Layers are independent, so
+// they are split into groups that run the whole pipeline on streams of their own: one group's
+// latency-bound kernels then overlap the other groups' bandwidth- and ALU-bound ones.
+constexpr int kMaxGroups = 4;
+
+static int layer_groups(int L) {
+    int g = kMaxGroups;
+    const char* e = getenv("ZIPLM_LAYER_GROUPS");
+    if (e) g = atoi(e);
+    if (g < 1) g = 1;
+    if (g > kMaxGroups) g = kMaxGroups;
+    if (g > L) g = L;
+    return g;
+}
+
+static int group_begin(int L, int groups, int g) { return (int)((long long)L * g / groups); }
+
+static size_t grouped_lazy_bytes(int L, int r, int d, int n_levels, int groups) {
+    size_t b = 0;
+    for (int g = 0; g < groups; ++g)
+        b += lazy_workspace_bytes(group_begin(L, groups, g + 1) - group_begin(L, groups, g), r, d,
+                                  n_levels);
+    return b;
+}
+
+// Internal streams, created once per device and kept for the life of the process.
+static cudaStream_t* group_streams() {
+    static cudaStream_t pool[64][kMaxGroups] = {};
+    static bool ready[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ready[dev]) {
+        for (int g = 0; g < kMaxGroups; ++g)
+            if (cudaStreamCreateWithFlags(&pool[dev][g], cudaStreamNonBlocking) != cudaSuccess)
+                return nullptr;
+        ready[dev] = true;
+    }
+    return pool[dev];
+}
+
 size_t neuron_workspace_bytes(int L, int r, int d, int n_levels) {
     const size_t a = carve_neuron(nullptr, L, r, d).total;
-    const size_t b = lazy_path_supported(d) ? lazy_workspace_bytes(L, r, d, n_levels) : 0;
+    size_t b = 0;
+    if (lazy_path_supported(d))   // every group count up to the maximum must fit
+        for (int g = 1; g <= kMaxGroups && g <= L; ++g) {
+            const size_t t = grouped_lazy_bytes(L, r, d, n_levels, g);
+            if (t > b) b = t;
+        }
     return a > b ? a : b;
+}
+
+static ziplm_status run_prune_lazy_grouped(const float* W, const float* H, int L, int r, int d,
+                                           float damp_frac, const int* levels, int n_levels,
+                                           float* W_snap, float* loss, float* base_loss, int* order,
+                                           float* saliency, int* layer_status, void* ws,
+                                           cudaStream_t st) {
+    const int groups = layer_groups(L);
+    cudaStream_t* pool = groups > 1 ? group_streams() : nullptr;
+    if (groups <= 1 || !pool)
+        return run_prune_lazy(W, H, L, r, d, damp_frac, levels, n_levels, W_snap, loss, base_loss,
+                              order, saliency, layer_status, ws,
+                              lazy_workspace_bytes(L, r, d, n_levels), st);
+    cudaEvent_t fork, join[kMaxGroups];
+    ZIPLM_CHECK_CUDA(cudaEventCreateWithFlags(&fork, cudaEventDisableTiming));
+    ZIPLM_CHECK_CUDA(cudaEventRecord(fork, st));
+    ziplm_status rc = ZIPLM_OK;
+    char* wsp = static_cast<char*>(ws);
+    for (int g = 0; g < groups; ++g) {
+        const int l0 = group_begin(L, groups, g), Lg = group_begin(L, groups, g + 1) - l0;
+        const size_t bytes = lazy_workspace_bytes(Lg, r, d, n_levels);
+        cudaStream_t sg = pool[g];
+        bool ok = cudaStreamWaitEvent(sg, fork, 0) == cudaSuccess;
+        if (ok && rc == ZIPLM_OK)
+            rc = run_prune_lazy(W + (size_t)l0 * r * d, H + (size_t)l0 * d * d, Lg, r, d, damp_frac,
+                                levels, n_levels, W_snap + (size_t)l0 * n_levels * r * d,
+                                loss + (size_t)l0 * n_levels, base_loss ? base_loss + l0 : nullptr,
+                                order + (size_t)l0 * d, saliency ? saliency + (size_t)l0 * d : nullptr,
+                                layer_status + l0, wsp, bytes, sg);
+        // always join, so that the caller's stream stays ordered after whatever was enqueued
+        ok = ok && cudaEventCreateWithFlags(&join[g], cudaEventDisableTiming) == cudaSuccess;
+        if (ok) {
+            ok = cudaEventRecord(join[g], sg) == cudaSuccess &&
+                 cudaStreamWaitEvent(st, join[g], 0) == cudaSuccess;
+            cudaEventDestroy(join[g]);
+        }
+        if (!ok && rc == ZIPLM_OK) rc = ZIPLM_ERR_CUDA;
+        wsp += bytes;
+    }
+    cudaEventDestroy(fork);
+    return rc;
 }
 
 ziplm_status run_prune_neurons(const float* W, const float* H, int L, int r, int d,
@@ -396,8 +483,8 @@ ziplm_status run_prune_neurons(const float* W, const float* H, int L, int r, int
                                int* layer_status, void* ws, size_t ws_bytes, cudaStream_t st) {
     if (ws_bytes < neuron_workspace_bytes(L, r, d, n_levels)) return ZIPLM_ERR_WORKSPACE;
     if (use_lazy_path(d))
-        return run_prune_lazy(W, H, L, r, d, damp_frac, levels, n_levels, W_snap, loss, base_loss,
-                              order, saliency, layer_status, ws, ws_bytes, st);
+        return run_prune_lazy_grouped(W, H, L, r, d, damp_frac, levels, n_levels, W_snap, loss,
+                                      base_loss, order, saliency, layer_status, ws, st);
     NeuronWs w = carve_neuron(ws, L, r, d);
     const int G = d;
 

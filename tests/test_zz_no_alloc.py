@@ -28,7 +28,7 @@ def test_noalloc_inverse_matches_the_workspace_version_twice_in_a_row():
     import paper_2302_04089_b200 as z
     for d, L, shift in ((320, 4, 0), (200, 2, 50)):
         H = make_h(d, L, shift)
-        assert z.inverse_workspace_bytes(L, d) <= 8 << 20
+        assert z.inverse_workspace_bytes(L, d) <= 12 << 20
         ref, ref_status = z.damped_inverse(H, 0.01)
         got = torch.full((L, d, d), float("nan"), dtype=torch.float64, device="cuda")
         status = torch.full((L,), -7, dtype=torch.int32, device="cuda")
@@ -46,7 +46,7 @@ def test_noalloc_inverse_matches_the_workspace_version_twice_in_a_row():
 def test_noalloc_inverse_rejects_requests_beyond_its_scratch():
     import paper_2302_04089_b200 as z
     d, L = 768, 1
-    assert z.inverse_workspace_bytes(L, d) > 8 << 20
+    assert z.inverse_workspace_bytes(L, d) > 12 << 20
     H = torch.eye(d, device="cuda")[None].contiguous()
     out = torch.zeros(L, d, d, dtype=torch.float64, device="cuda")
     status = torch.zeros(L, dtype=torch.int32, device="cuda")
