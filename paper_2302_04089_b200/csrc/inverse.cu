@@ -24,26 +24,39 @@ static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratch
 
 namespace ziplm {
 namespace {
-constexpr int KC = 16;          // k-chunk staged in shared memory per iteration
-constexpr int LDS = kTile + 2;  // padded shared-memory row length (doubles)
-constexpr int GT = 128;         // threads of a product CTA: 8 x 4 outputs per thread
+constexpr int KC = 8;           // k-chunk staged in shared memory per iteration
+constexpr int LDS = kTile + 2;  // padded shared-memory row length (doubles), keeps rows 16-byte aligned
+constexpr int GT = 64;          // threads of a product CTA: 8 x 8 outputs per thread
 
+// Both operands sit in shared memory k-major (s[k][i]): the inner loop then reads two
+// neighbouring rows / columns per 128-bit load, 8 loads for 64 FMAs.
 struct TileSmem {
     double a[2][KC][LDS];
     double b[2][KC][LDS];
 };
 
-// Fetch one 64 x KC chunk of an operand into registers (8 doubles per thread).
-//   T == false: stored 64 x K row-major (op(i,k) = P[i*ld + k]); true: stored K x 64.
+// Fetch one 64 x KC chunk of an operand into registers (8 doubles per thread) and put it into
+// shared memory as s[k][i].
+//   T == false: stored 64 x K row-major (op(i,k) = P[i*ld + k]): a thread takes one row's 8 k's
+//               and writes them down a column of s (consecutive threads -> consecutive i);
+//   T == true : stored K x 64 (op(i,k) = P[k*ld + i]): a thread takes pairs along i.
 template <bool T>
 __device__ __forceinline__ void chunk_load(double (&r)[8], const double* P, int ld, int k0) {
     const int tid = threadIdx.x;
-    const double* src = T ? P + (size_t)(k0 + (tid >> 3)) * ld + (tid & 7) * 8
-                          : P + (size_t)(tid >> 1) * ld + k0 + (tid & 1) * 8;
+    if (T) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const double2 v = *reinterpret_cast<const double2*>(src + 2 * e);
-        r[2 * e] = v.x; r[2 * e + 1] = v.y;
+        for (int e = 0; e < 4; ++e) {
+            const double2 v = *reinterpret_cast<const double2*>(
+                P + (size_t)(k0 + (tid >> 5) + 2 * e) * ld + (tid & 31) * 2);
+            r[2 * e] = v.x; r[2 * e + 1] = v.y;
+        }
+    } else {
+        const double* src = P + (size_t)tid * ld + k0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const double2 v = *reinterpret_cast<const double2*>(src + 2 * e);
+            r[2 * e] = v.x; r[2 * e + 1] = v.y;
+        }
     }
 }
 
@@ -51,66 +64,75 @@ template <bool T>
 __device__ __forceinline__ void chunk_store(double (*s)[LDS], const double (&r)[8]) {
     const int tid = threadIdx.x;
     if (T) {
-        const int kk = tid >> 3, iq = (tid & 7) * 8;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) s[kk][iq + e] = r[e];
+        for (int e = 0; e < 4; ++e)
+            *reinterpret_cast<double2*>(&s[(tid >> 5) + 2 * e][(tid & 31) * 2]) =
+                make_double2(r[2 * e], r[2 * e + 1]);
     } else {
-        const int i = tid >> 1, kq = (tid & 1) * 8;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) s[kq + e][i] = r[e];
+        for (int e = 0; e < 8; ++e) s[e][tid] = r[e];
     }
 }
 
-// acc(64x64) += opA(64xK) * opB(Kx64); 128 threads, thread (ty,tx) owns rows ty+8a (a < 8) and
-// cols tx+16b (b < 4).  The next chunk is fetched into registers while the current one is
-// multiplied out of shared memory (two buffers, one barrier per chunk).  The operand pointers
-// are deliberately not __restrict__: callers may read tiles written earlier in the same launch
-// sequence.  Ends with __syncthreads().
+// Row / column of output element (p, q) of thread (ty, tx): pairs of neighbours, 16 apart.
+__device__ __forceinline__ int own_index(int t, int p) { return 2 * t + 16 * (p >> 1) + (p & 1); }
+
+// acc(64x64) += opA(64xK) * opB(Kx64); 64 threads, thread (ty,tx) = (tid/8, tid%8) owns the rows
+// own_index(ty, p) and the columns own_index(tx, q), p, q < 8.  The next chunk is fetched into
+// registers while the current one is multiplied out of shared memory (two buffers, one barrier
+// per chunk).  The operand pointers are deliberately not __restrict__: callers may read tiles
+// written earlier in the same launch sequence.  Ends with __syncthreads().
+//   TA == false: A stored 64 x K row-major; true: stored K x 64.
+//   TB == false: B stored K x 64 row-major; true: stored 64 x K.
 template <bool TA, bool TB>
-__device__ __forceinline__ void dgemm_tile(double (&acc)[8][4], const double* A, int lda,
+__device__ __forceinline__ void dgemm_tile(double (&acc)[8][8], const double* A, int lda,
                                            const double* B, int ldb, int K, TileSmem& sm) {
     const int tid = threadIdx.x;
-    const int ty = tid >> 4, tx = tid & 15;
+    const int ty = tid >> 3, tx = tid & 7;
     if (K <= 0) return;
+    constexpr bool LA = TA, LB = !TB;       // loader orientation: true = stored K x 64
     double ra[8], rb[8];
-    chunk_load<TA>(ra, A, lda, 0);
-    chunk_load<TB ? false : true>(rb, B, ldb, 0);
-    chunk_store<TA>(sm.a[0], ra);
-    chunk_store<TB ? false : true>(sm.b[0], rb);
+    chunk_load<LA>(ra, A, lda, 0);
+    chunk_load<LB>(rb, B, ldb, 0);
+    chunk_store<LA>(sm.a[0], ra);
+    chunk_store<LB>(sm.b[0], rb);
     __syncthreads();
     int buf = 0;
     for (int k0 = 0; k0 < K; k0 += KC) {
         const bool more = k0 + KC < K;
         if (more) {
-            chunk_load<TA>(ra, A, lda, k0 + KC);
-            chunk_load<TB ? false : true>(rb, B, ldb, k0 + KC);
+            chunk_load<LA>(ra, A, lda, k0 + KC);
+            chunk_load<LB>(rb, B, ldb, k0 + KC);
         }
 #pragma unroll
         for (int kk = 0; kk < KC; ++kk) {
-            double a[8], b[4];
+            double a[8], b[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) a[q] = sm.a[buf][kk][ty + 8 * q];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) b[q] = sm.b[buf][kk][tx + 16 * q];
+            for (int q = 0; q < 4; ++q) {
+                const double2 va = *reinterpret_cast<const double2*>(&sm.a[buf][kk][2 * ty + 16 * q]);
+                const double2 vb = *reinterpret_cast<const double2*>(&sm.b[buf][kk][2 * tx + 16 * q]);
+                a[2 * q] = va.x; a[2 * q + 1] = va.y;
+                b[2 * q] = vb.x; b[2 * q + 1] = vb.y;
+            }
 #pragma unroll
             for (int p = 0; p < 8; ++p)
 #pragma unroll
-                for (int q = 0; q < 4; ++q) acc[p][q] = fma(a[p], b[q], acc[p][q]);
+                for (int q = 0; q < 8; ++q) acc[p][q] = fma(a[p], b[q], acc[p][q]);
         }
         if (more) {
-            chunk_store<TA>(sm.a[buf ^ 1], ra);
-            chunk_store<TB ? false : true>(sm.b[buf ^ 1], rb);
+            chunk_store<LA>(sm.a[buf ^ 1], ra);
+            chunk_store<LB>(sm.b[buf ^ 1], rb);
         }
         __syncthreads();
         buf ^= 1;
     }
 }
 
-__device__ __forceinline__ void zero_acc(double (&acc)[8][4]) {
+__device__ __forceinline__ void zero_acc(double (&acc)[8][8]) {
 #pragma unroll
     for (int p = 0; p < 8; ++p)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[p][q] = 0.0;
+        for (int q = 0; q < 8; ++q) acc[p][q] = 0.0;
 }
 
 // lambda[l] = damp_frac * mean(diag H[l]); flags non-finite diagonals and non-positive means.
@@ -214,18 +236,19 @@ __global__ void __launch_bounds__(GT) k_dgemm_tiles(GemmTask t, int dp) {
                                       : ((size_t)(t.a_r + ti) * kTile * dp + (size_t)(t.a_c + klo) * kTile));
     const double* B = t.B + lay + (TB ? ((size_t)(t.b_r + tj) * kTile * dp + (size_t)(t.b_c + klo) * kTile)
                                       : ((size_t)(t.b_r + klo) * kTile * dp + (size_t)(t.b_c + tj) * kTile));
-    double acc[8][4];
+    double acc[8][8];
     zero_acc(acc);
     dgemm_tile<TA, TB>(acc, A, dp, B, dp, (khi - klo) * kTile, sm);
     double* out = t.C + lay + (size_t)(t.c_r + ti) * kTile * dp + (size_t)(t.c_c + tj) * kTile;
-    const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+    const int ty = threadIdx.x >> 3, tx = threadIdx.x & 7;
 #pragma unroll
     for (int p = 0; p < 8; ++p)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            double* o = out + (size_t)(ty + 8 * p) * dp + tx + 16 * q;
-            const double v = t.alpha * acc[p][q];
-            *o = t.beta ? (*o + v) : v;
+        for (int q = 0; q < 8; q += 2) {
+            double2* o = reinterpret_cast<double2*>(out + (size_t)own_index(ty, p) * dp + own_index(tx, q));
+            double2 v = make_double2(t.alpha * acc[p][q], t.alpha * acc[p][q + 1]);
+            if (t.beta) { const double2 c = *o; v.x += c.x; v.y += c.y; }
+            *o = v;
         }
 }
 
@@ -244,16 +267,16 @@ __global__ void __launch_bounds__(256) k_potf2(const double* A, double* F, doubl
         s[e >> 6][e & 63] = A[off + (size_t)(e >> 6) * dp + (e & 63)];
     __syncthreads();
     for (int c = 0; c < kTile; ++c) {
-        if (tid == 0) {
-            double p = s[c][c];
-            if (!(p > 0.0) || !isfinite(p)) {   // not positive definite (or NaN): flag, keep going
-                if (!sflag) sflag = isfinite(p) ? ZIPLM_ERR_NOT_PD : ZIPLM_ERR_NONFINITE;
-                p = 1.0;
-            }
-            s[c][c] = sqrt(p);
+        // every thread forms 1/sqrt(pivot) itself: no broadcast, two barriers per column
+        double p = s[c][c];
+        if (!(p > 0.0) || !isfinite(p)) {   // not positive definite (or NaN): flag, keep going
+            if (tid == 0 && !sflag) sflag = isfinite(p) ? ZIPLM_ERR_NOT_PD : ZIPLM_ERR_NONFINITE;
+            p = 1.0;
         }
-        __syncthreads();
-        if (tid > c && tid < kTile) s[tid][c] /= s[c][c];
+        const double rinv = rsqrt(p);
+        __syncthreads();                    // all threads have read the pivot
+        if (tid == c) s[c][c] = p * rinv;
+        else if (tid > c && tid < kTile) s[tid][c] *= rinv;
         __syncthreads();
         // trailing update of the lower triangle: rows ty + 16a, cols tx + 16b
 #pragma unroll
@@ -308,16 +331,16 @@ __global__ void __launch_bounds__(GT) k_lauum(const double* M, int dp, int T, in
     while (rem > i) { rem -= i + 1; ++i; }
     const int j = rem;
     const double* Ml = M + (size_t)l * dp * dp;
-    double acc[8][4];
+    double acc[8][8];
     zero_acc(acc);
     dgemm_tile<true, false>(acc, Ml + (size_t)i * kTile * dp + (size_t)i * kTile, dp,
                             Ml + (size_t)i * kTile * dp + (size_t)j * kTile, dp, (T - i) * kTile, sm);
-    const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+    const int ty = threadIdx.x >> 3, tx = threadIdx.x & 7;
 #pragma unroll
     for (int p = 0; p < 8; ++p)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int row = i * kTile + ty + 8 * p, col = j * kTile + tx + 16 * q;
+        for (int q = 0; q < 8; ++q) {
+            const int row = i * kTile + own_index(ty, p), col = j * kTile + own_index(tx, q);
             if (row >= d || col >= d) continue;
             const double v = acc[p][q];
             if (out64 && row >= col) {
