@@ -304,13 +304,15 @@ def run_ours(args, shape):
     step()
     torch.cuda.synchronize()
     phases = z.profile_end()
-    os.environ["ZIPLM_NEURON_PATH"] = "stream"
-    step()
-    z.profile_begin()
-    step()
-    torch.cuda.synchronize()
-    phases_stream = z.profile_end()
-    del os.environ["ZIPLM_NEURON_PATH"]
+    phases_stream = {"update": (0.0, 0)}
+    if not args.skip_stream_leg:
+        os.environ["ZIPLM_NEURON_PATH"] = "stream"
+        step()
+        z.profile_begin()
+        step()
+        torch.cuda.synchronize()
+        phases_stream = z.profile_end()
+        del os.environ["ZIPLM_NEURON_PATH"]
     del os.environ["ZIPLM_LAYER_GROUPS"]
 
     if dist is not None:
@@ -391,6 +393,8 @@ def main():
     ap.add_argument("--max-removed", type=int, default=0,
                     help="profiling aid: stop the greedy loop after this many removals")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling aid: no host-buffer leg")
+    ap.add_argument("--skip-stream-leg", action="store_true",
+                    help="profiling aid: do not time the per-step streaming variant")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     shape = wl.CONFIGS[WORKLOAD][0]
