@@ -169,6 +169,19 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in prune_lazy.cu)
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu captures
+# summarised under profiles/ (taken on 4 of the 12 layers and scaled by 3: traffic grows in
+# proportion to the layers).  Only valid for the bench workload; the kernels have not changed
+# since the captures.
+NCU_TRAFFIC = {
+    # k_lazy_update_aq, first block (n_new = 3040): profiles/k_lazy_kernels_c3_4layers.md
+    "k_lazy_update_aq": dict(bytes=3 * (161.9e6 + 93.5e6), launch="n_new = 3040, m = 32",
+                             algorithmic=12 * 16.0 * 3040 * 3039 / 2),
+    # k_neuron_update at n = 3066: profiles/k_neuron_update_c3_4layers.md
+    "k_neuron_update": dict(bytes=3 * (113.8e6 + 56.6e6), launch="n = 3066",
+                            algorithmic=12 * (8.0 * 768 * 3066 + 4.0 * 3066 * 3066)),
+}
+
 
 def lazy_update_work(L, G, levels):
     """Algorithmic work of k_lazy_update_aq over one greedy run: a launch that leaves n live
@@ -315,16 +328,15 @@ def run_ours(args, shape):
         del os.environ["ZIPLM_NEURON_PATH"]
     del os.environ["ZIPLM_LAYER_GROUPS"]
 
-    if dist is not None:
-        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    from paper_2302_04089_b200.parallel import max_over_ranks
+    ms, ms_e2e = max_over_ranks(ms), max_over_ranks(ms_e2e)
     n_removed = G - min(levels)
     structures = world * L * n_removed
     value = structures / (ms * 1e-3)
     e2e_value = structures / (ms_e2e * 1e-3)
 
     if rank == 0:
+        full_workload = args.layers == 0 and args.max_removed == 0
         peak, peak_src = load_peaks()
         upd_ms, upd_n = phases_stream["update"]
         alg_bytes, n_launch = update_bytes(L, r, G, n_removed)
@@ -352,7 +364,9 @@ def run_ours(args, shape):
             gpu_launches=int(launches),
             clocks=clocks,
             roofline=dict(kernel="k_lazy_update_aq", bound="hbm", achieved=aq_gbs, peak=peak,
-                          unit="GB/s", frac=aq_gbs / peak, traffic=None, peak_source=peak_src,
+                          unit="GB/s", frac=aq_gbs / peak,
+                          traffic=NCU_TRAFFIC["k_lazy_update_aq"]["bytes"] if full_workload else None,
+                          traffic_note=NCU_TRAFFIC["k_lazy_update_aq"], peak_source=peak_src,
                           launches=aq_n, avg_launch_us=1e3 * aq_ms / max(aq_n, 1),
                           algorithmic_bytes_per_step=aq_bytes,
                           alu=dict(achieved_tfma=aq_fma / (aq_ms * 1e-3) / 1e12 if aq_ms > 0 else 0.0,
@@ -362,7 +376,9 @@ def run_ours(args, shape):
                                         "= 74.4)")),
             roofline_streaming_update=dict(
                 kernel="k_neuron_update", bound="hbm", achieved=achieved, peak=peak, unit="GB/s",
-                frac=achieved / peak, traffic=None, peak_source=peak_src, launches=upd_n,
+                frac=achieved / peak,
+                traffic=NCU_TRAFFIC["k_neuron_update"]["bytes"] if full_workload else None,
+                traffic_note=NCU_TRAFFIC["k_neuron_update"], peak_source=peak_src, launches=upd_n,
                 avg_launch_us=1e3 * upd_ms / max(upd_n, 1), algorithmic_bytes_per_step=alg_bytes,
                 note="per-step fused H^-1/W update of the streaming variant "
                      "(ZIPLM_NEURON_PATH=stream), timed in a separate step",
