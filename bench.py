@@ -352,7 +352,7 @@ def run_ours(args, shape):
             config=dict(workload=WORKLOAD if (args.layers == 0 and args.max_removed == 0)
                         else WORKLOAD + " (reduced: profiling aid)", layers=L, d_row=r, d_col=d, n_tokens=N, group_size=g,
                         levels=len(levels), damp_frac=shape.damp_frac,
-                        l2_policy="inputs_exceed_l2 (X 2.4 GB, H^-1 workspace 0.45 GB per step)",
+                        l2_policy="inputs_exceed_l2 (X 2.4 GB and about 2 GB of loop state per step)",
                         parallelism=f"layer-sharded x{world}, no collective"),
             layers_per_sec=world * L / (ms * 1e-3),
             phases_ms={k: round(v[0], 3) for k, v in phases.items() if v[1] > 0},
@@ -399,7 +399,7 @@ def run_ours(args, shape):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-steps", type=int, default=24)
