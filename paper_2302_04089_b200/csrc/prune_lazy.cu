@@ -112,17 +112,39 @@ __device__ __forceinline__ bool better(const Cand& x, const Cand& y) {   // x st
     return lhs < rhs || (lhs == rhs && x.org < y.org);
 }
 
-__device__ __forceinline__ Cand shfl_cand(const Cand& c, int off) {
+__device__ __forceinline__ void merge_cand(Cand& best, const Cand& o) {
+    if (o.pos >= 0 && (best.pos < 0 || better(o, best))) best = o;
+}
+
+__device__ __forceinline__ Cand bcast_cand(const Cand& c, int src_lane) {
     Cand o;
-    o.a = __shfl_xor_sync(0xffffffffu, c.a, off);
-    o.q = __shfl_xor_sync(0xffffffffu, c.q, off);
-    o.org = __shfl_xor_sync(0xffffffffu, c.org, off);
-    o.pos = __shfl_xor_sync(0xffffffffu, c.pos, off);
+    o.a = __shfl_sync(0xffffffffu, c.a, src_lane);
+    o.q = __shfl_sync(0xffffffffu, c.q, src_lane);
+    o.org = __shfl_sync(0xffffffffu, c.org, src_lane);
+    o.pos = __shfl_sync(0xffffffffu, c.pos, src_lane);
     return o;
 }
 
-__device__ __forceinline__ void merge_cand(Cand& best, const Cand& o) {
-    if (o.pos >= 0 && (best.pos < 0 || better(o, best))) best = o;
+// Best candidate of a warp (every lane returns it).  A cheap fp32 quotient orders the lanes; only
+// the lanes within 1e-5 of the fp32 minimum (almost always a single one) go through the exact
+// float64 comparison, so the common case costs six 32-bit shuffles instead of five rounds of
+// 64-bit exchanges.
+__device__ __forceinline__ Cand warp_best(const Cand& mine) {
+    float r = INFINITY;
+    if (mine.pos >= 0) r = cand_valid(mine) ? (float)mine.q / (float)mine.a : -INFINITY;
+    float rmin = r;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) rmin = fminf(rmin, __shfl_xor_sync(0xffffffffu, rmin, off));
+    const bool near_min = mine.pos >= 0 && (r == rmin || r <= rmin + fabsf(rmin) * 1e-5f);
+    unsigned mask = __ballot_sync(0xffffffffu, near_min);
+    Cand best;
+    best.a = 1.0; best.q = 0.0; best.org = 0x7fffffff; best.pos = -1;
+    while (mask) {
+        const int b = __ffs(mask) - 1;
+        mask &= mask - 1;
+        merge_cand(best, bcast_cand(mine, b));
+    }
+    return best;
 }
 
 // nsteps greedy steps of one layer, run by a thread-block cluster of CS CTAs (CS = 1, 2, 4 or 8,
@@ -201,8 +223,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
             c.a = da[e]; c.q = dq[e]; c.org = org[e]; c.pos = k0 + e;
             merge_cand(best, c);
         }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) merge_cand(best, shfl_cand(best, off));
+        best = warp_best(best);
         if (lane == 0) s_cand[par][warp] = best;
         cluster.sync();
         // ---- warp 0 of every CTA: global pick from all warps of all CTAs, then the pending
@@ -214,15 +235,14 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
                 const Cand* remote = cluster.map_shared_rank(&s_cand[par][e % NW], e / NW);
                 merge_cand(g, *remote);
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) merge_cand(g, shfl_cand(g, off));
+            g = warp_best(g);
             int p = g.pos;
             if (p < 0) p = 0;
             double h = g.a;
             int bad = 0;
             if (!isfinite(g.q) || !isfinite(h)) { bad = ZIPLM_ERR_NONFINITE; h = 1.0; }
             else if (!(h > 0.0)) { bad = ZIPLM_ERR_NOT_PD; h = 1.0; }
-            const double rs = 1.0 / sqrt(h);
+            const double rs = rsqrt(h);
             const int prow = p / S, pl = p - prow * S;
             float up = 0.f, zp = 0.f;
             if (lane < m) {
@@ -235,11 +255,11 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
             if (lane == 0) {
                 s_p = p;
                 s_rs = rs;
-                s_half = g.q / (2.0 * h);
+                s_half = 0.5 * g.q * rs * rs;
                 s_pm[m] = p;
                 s_rsm[m] = rs;
                 if (rank == 0) {
-                    const double rho = bad ? 0.0 : g.q / h;
+                    const double rho = bad ? 0.0 : g.q * rs * rs;
                     if (bad) set_layer_status(layer_status, l, bad);
                     sumrho += rho;
                     order[(size_t)l * G + t0 + m] = g.org;
@@ -252,28 +272,30 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
         const double rs = s_rs, half = s_half;
         // ---- true pivot columns of H^-1 and Q on the owned positions; float64 diagonal downdate
         if (owner_thread) {
-            double a[4], q[4];
+            // The pending terms are subtracted with fp32 FMAs, one rounding per term: exactly
+            // what the per-step streaming variant does to the stored entry.
+            float a[4], q[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int k = k0 + e;
-                a[e] = 0.0; q[e] = 0.0;
+                a[e] = 0.f; q[e] = 0.f;
                 if (alive[e] && k != p) {
                     const size_t off = (k < p) ? ((size_t)p * d + k) : ((size_t)k * d + p);
-                    a[e] = (double)Al[off];
-                    q[e] = (double)Ql[off];
+                    a[e] = Al[off];
+                    q[e] = Ql[off];
                 }
             }
 #pragma unroll 4
             for (int s = 0; s < m; ++s) {
                 const float4 u4 = *reinterpret_cast<const float4*>(sU + (size_t)s * S + kloc);
                 const float4 z4 = *reinterpret_cast<const float4*>(sZ + (size_t)s * S + kloc);
-                const double up = (double)sUp[s], zp = (double)sZp[s];
+                const float up = sUp[s], zp = sZp[s];
                 const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, zz[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    a[e] = fma(-(double)uu[e], up, a[e]);
-                    q[e] = fma(-(double)zz[e], up, q[e]);
-                    q[e] = fma(-(double)uu[e], zp, q[e]);
+                    a[e] = fmaf(-uu[e], up, a[e]);
+                    q[e] = fmaf(-zz[e], up, q[e]);
+                    q[e] = fmaf(-uu[e], zp, q[e]);
                 }
             }
             float u32[4], z32[4];
@@ -282,8 +304,8 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
                 const int k = k0 + e;
                 u32[e] = 0.f; z32[e] = 0.f;
                 if (alive[e] && k != p) {
-                    const double u = a[e] * rs;
-                    const double z = q[e] * rs - half * u;
+                    const double u = (double)a[e] * rs;
+                    const double z = (double)q[e] * rs - half * u;
                     da[e] -= u * u;
                     dq[e] -= 2.0 * z * u;
                     u32[e] = (float)u;
@@ -313,10 +335,11 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
                 w[m] = (m < nsteps && i < r) ? Wl[(size_t)s_pm[m] * rp + i] : 0.f;
 #pragma unroll
             for (int m = 0; m < BMAX; ++m) {
-                double acc = (double)w[m];
+                double acc[4] = {(double)w[m], 0.0, 0.0, 0.0};
 #pragma unroll
-                for (int s = 0; s < m; ++s) acc = fma(-(double)c[s], (double)sT[m][s], acc);
-                c[m] = (m < nsteps) ? (float)(acc * s_rsm[m]) : 0.f;
+                for (int s = 0; s < m; ++s)
+                    acc[s & 3] = fma(-(double)c[s], (double)sT[m][s], acc[s & 3]);
+                c[m] = (m < nsteps) ? (float)(((acc[0] + acc[1]) + (acc[2] + acc[3])) * s_rsm[m]) : 0.f;
                 if (m < nsteps) Cl[(size_t)m * rp + i] = c[m];
             }
         }
