@@ -294,10 +294,11 @@ __global__ void __launch_bounds__(256) k_potf2(const double* A, double* F, doubl
     }
     // inverse of the lower-triangular factor: thread `cidx` builds column cidx by forward
     // substitution.  Entry (i, cidx), i > cidx, is parked transposed in the unused strict upper
-    // triangle of s (slot [cidx][i]); the diagonal goes to dinv.
+    // triangle of s (slot [cidx][i]); the reciprocal diagonal goes to dinv first.
+    if (tid < kTile) dinv[tid] = 1.0 / s[tid][tid];
+    __syncthreads();
     if (tid < kTile) {
         const int cidx = tid;
-        dinv[cidx] = 1.0 / s[cidx][cidx];
         for (int i = cidx + 1; i < kTile; ++i) {
             double a0 = -s[i][cidx] * dinv[cidx], a1 = 0.0, a2 = 0.0, a3 = 0.0;
             int k = cidx + 1;
@@ -308,7 +309,7 @@ __global__ void __launch_bounds__(256) k_potf2(const double* A, double* F, doubl
                 a3 = fma(-s[i][k + 3], s[cidx][k + 3], a3);
             }
             for (; k < i; ++k) a0 = fma(-s[i][k], s[cidx][k], a0);
-            s[cidx][i] = ((a0 + a1) + (a2 + a3)) / s[i][i];
+            s[cidx][i] = ((a0 + a1) + (a2 + a3)) * dinv[i];
         }
     }
     __syncthreads();
@@ -367,6 +368,7 @@ template <bool TA, bool TB>
 ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
     const int tiles = t.lower_only ? t.mt * (t.mt + 1) / 2 : t.mt * t.nt;
     if (tiles <= 0 || t.kt <= 0) return ZIPLM_OK;
+    PhaseScope ps(PH_INV_PRODUCTS, c.st);
     k_dgemm_tiles<TA, TB><<<dim3(tiles, c.L), GT, 0, c.st>>>(t, c.dp);
     ZIPLM_CHECK_LAUNCH();
     return ZIPLM_OK;
@@ -376,6 +378,7 @@ ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
 // and M its inverse.
 ziplm_status factor_range(const InvCtx& c, int lo, int hi) {
     if (hi - lo == 1) {
+        PhaseScope ps(PH_INV_LEAVES, c.st);
         k_potf2<<<c.L, 256, 0, c.st>>>(c.A, c.F, c.M, c.dp, lo, c.layer_status);
         ZIPLM_CHECK_LAUNCH();
         return ZIPLM_OK;
@@ -431,8 +434,11 @@ ziplm_status run_damped_inverse(const float* H, int L, int d, float damp_frac, d
     ZIPLM_CHECK_LAUNCH();
     ziplm_status s = factor_range(ctx, 0, T);
     if (s != ZIPLM_OK) return s;
-    k_lauum<<<dim3(T * (T + 1) / 2, L), GT, 0, st>>>(ctx.M, dp, T, d, out64, tri32, pitch32, diag64);
-    ZIPLM_CHECK_LAUNCH();
+    {
+        PhaseScope ps(PH_INV_LAUUM, st);
+        k_lauum<<<dim3(T * (T + 1) / 2, L), GT, 0, st>>>(ctx.M, dp, T, d, out64, tri32, pitch32, diag64);
+        ZIPLM_CHECK_LAUNCH();
+    }
     if (lam_out) {
         ZIPLM_CHECK_CUDA(cudaMemcpyAsync(lam_out, lam, sizeof(double) * L, cudaMemcpyDeviceToDevice, st));
     }

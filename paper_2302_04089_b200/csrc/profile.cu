@@ -18,7 +18,8 @@ bool g_on = false;
 std::vector<Span> g_spans;
 const char* kPhaseNames[PH_COUNT] = {"hessian", "inverse", "init", "prep", "update", "snapshot",
                                      "block_score", "block_update", "lazy_steps", "lazy_update_aq",
-                                     "lazy_update_w"};
+                                     "lazy_update_w", "inverse_products", "inverse_leaves",
+                                     "inverse_lauum"};
 }  // namespace
 
 PhaseScope::PhaseScope(int phase, cudaStream_t st) : st_(st), idx_(-1) {
