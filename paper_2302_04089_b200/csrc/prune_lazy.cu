@@ -383,62 +383,81 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
 // Rank-m update of the strict lower triangles of H^-1 and Q with compaction (out of place):
 //   A'[i,j] = A[si,sj] - sum_s U[s,si] U[s,sj],
 //   Q'[i,j] = Q[si,sj] - sum_s (Z[s,si] U[s,sj] + U[s,si] Z[s,sj]),    si = src[i] > sj = src[j].
-// 64 x 64 tiles of the new index space, 4 x 4 elements per thread.
-__global__ void __launch_bounds__(256) k_lazy_update_aq(int n_new, int m, int d,
+// 64 x 64 tiles of the new index space, 128 threads, 8 rows x 4 columns of both matrices per
+// thread: per pending step six 128-bit shared-memory loads feed 96 FMAs.  Entries above the
+// diagonal of a tile that straddles it are written too (the upper triangles are never read).
+__global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
                                                         const float* __restrict__ A,
                                                         const float* __restrict__ Q,
                                                         float* __restrict__ A2, float* __restrict__ Q2,
                                                         const int* __restrict__ src,
                                                         const float* __restrict__ U,
                                                         const float* __restrict__ Z) {
-    __shared__ float sUr[BMAX][64], sZr[BMAX][64], sUc[BMAX][64], sZc[BMAX][64];
+    __shared__ __align__(16) float sUr[BMAX][64];
+    __shared__ __align__(16) float sZr[BMAX][64];
+    __shared__ __align__(16) float sUc[BMAX][64];
+    __shared__ __align__(16) float sZc[BMAX][64];
     __shared__ int srow[64], scol[64];
     const int l = blockIdx.y;
     int ti = 0, rem = blockIdx.x;
     while (rem > ti) { rem -= ti + 1; ++ti; }
     const int tj = rem;
     const int i0 = ti * 64, j0 = tj * 64;
-    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;     // rows 4ty + 32h + e, cols 4tx + e
     const int* sl = src + (size_t)l * d;
     if (tid < 64) srow[tid] = (i0 + tid < n_new) ? sl[i0 + tid] : -1;
-    else if (tid < 128) scol[tid - 64] = (j0 + tid - 64 < n_new) ? sl[j0 + tid - 64] : -1;
+    else scol[tid - 64] = (j0 + tid - 64 < n_new) ? sl[j0 + tid - 64] : -1;
     __syncthreads();
     const float* Ul = U + (size_t)l * BMAX * d;
     const float* Zl = Z + (size_t)l * BMAX * d;
-    for (int e = tid; e < m * 64; e += 256) {
-        const int s = e >> 6, c = e & 63;
-        const int sr = srow[c], sc = scol[c];
-        sUr[s][c] = sr >= 0 ? Ul[(size_t)s * d + sr] : 0.f;
-        sZr[s][c] = sr >= 0 ? Zl[(size_t)s * d + sr] : 0.f;
-        sUc[s][c] = sc >= 0 ? Ul[(size_t)s * d + sc] : 0.f;
-        sZc[s][c] = sc >= 0 ? Zl[(size_t)s * d + sc] : 0.f;
+    {
+        const int c = tid & 63;
+        const int idx = (tid < 64) ? srow[c] : scol[c];
+        float (*dU)[64] = (tid < 64) ? sUr : sUc;
+        float (*dZ)[64] = (tid < 64) ? sZr : sZc;
+#pragma unroll 4
+        for (int s = 0; s < m; ++s) {
+            dU[s][c] = idx >= 0 ? Ul[(size_t)s * d + idx] : 0.f;
+            dZ[s][c] = idx >= 0 ? Zl[(size_t)s * d + idx] : 0.f;
+        }
     }
     const float* Al = A + (size_t)l * d * d;
     const float* Ql = Q + (size_t)l * d * d;
-    float a[4][4], q[4][4];
+    int cs[4];
 #pragma unroll
-    for (int x = 0; x < 4; ++x)
+    for (int y = 0; y < 4; ++y) cs[y] = scol[4 * tx + y];
+    float a[8][4], q[8][4];
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const int il = 4 * ty + 32 * (x >> 2) + (x & 3), i = i0 + il;
+        const int sr = srow[il];
+        const size_t roff = (size_t)(sr >= 0 ? sr : 0) * d;
 #pragma unroll
         for (int y = 0; y < 4; ++y) {
-            const int i = i0 + ty + 16 * x, j = j0 + tx + 16 * y;
-            if (i < n_new && j < i) {
-                const size_t off = (size_t)srow[ty + 16 * x] * d + scol[tx + 16 * y];
-                a[x][y] = __ldcs(Al + off);
-                q[x][y] = __ldcs(Ql + off);
+            const int j = j0 + 4 * tx + y;
+            if (sr >= 0 && j < i) {
+                a[x][y] = __ldcs(Al + roff + cs[y]);
+                q[x][y] = __ldcs(Ql + roff + cs[y]);
             } else {
                 a[x][y] = 0.f; q[x][y] = 0.f;
             }
         }
+    }
     __syncthreads();
     for (int s = 0; s < m; ++s) {
-        float ur[4], zr[4], uc[4], zc[4];
+        float ur[8], zr[8];
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {
-            ur[x] = sUr[s][ty + 16 * x]; zr[x] = sZr[s][ty + 16 * x];
-            uc[x] = sUc[s][tx + 16 * x]; zc[x] = sZc[s][tx + 16 * x];
+        for (int h = 0; h < 2; ++h) {
+            const float4 v0 = *reinterpret_cast<const float4*>(&sUr[s][4 * ty + 32 * h]);
+            const float4 v1 = *reinterpret_cast<const float4*>(&sZr[s][4 * ty + 32 * h]);
+            ur[4 * h] = v0.x; ur[4 * h + 1] = v0.y; ur[4 * h + 2] = v0.z; ur[4 * h + 3] = v0.w;
+            zr[4 * h] = v1.x; zr[4 * h + 1] = v1.y; zr[4 * h + 2] = v1.z; zr[4 * h + 3] = v1.w;
         }
+        const float4 u4 = *reinterpret_cast<const float4*>(&sUc[s][4 * tx]);
+        const float4 z4 = *reinterpret_cast<const float4*>(&sZc[s][4 * tx]);
+        const float uc[4] = {u4.x, u4.y, u4.z, u4.w}, zc[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
-        for (int x = 0; x < 4; ++x)
+        for (int x = 0; x < 8; ++x)
 #pragma unroll
             for (int y = 0; y < 4; ++y) {
                 a[x][y] = fmaf(-ur[x], uc[y], a[x][y]);
@@ -448,16 +467,19 @@ __global__ void __launch_bounds__(256) k_lazy_update_aq(int n_new, int m, int d,
     }
     float* Ao = A2 + (size_t)l * d * d;
     float* Qo = Q2 + (size_t)l * d * d;
+    const int j = j0 + 4 * tx;
 #pragma unroll
-    for (int x = 0; x < 4; ++x)
-#pragma unroll
-        for (int y = 0; y < 4; ++y) {
-            const int i = i0 + ty + 16 * x, j = j0 + tx + 16 * y;
-            if (i < n_new && j < i) {
-                Ao[(size_t)i * d + j] = a[x][y];
-                Qo[(size_t)i * d + j] = q[x][y];
-            }
+    for (int x = 0; x < 8; ++x) {
+        const int i = i0 + 4 * ty + 32 * (x >> 2) + (x & 3);
+        if (i >= n_new || j >= i) continue;
+        if (j + 3 >= d) {
+            for (int e = 0; e < 4; ++e)
+                if (j + e < i) { Ao[(size_t)i * d + j + e] = a[x][e]; Qo[(size_t)i * d + j + e] = q[x][e]; }
+        } else {
+            *reinterpret_cast<float4*>(Ao + (size_t)i * d + j) = make_float4(a[x][0], a[x][1], a[x][2], a[x][3]);
+            *reinterpret_cast<float4*>(Qo + (size_t)i * d + j) = make_float4(q[x][0], q[x][1], q[x][2], q[x][3]);
         }
+    }
 }
 
 // Rank-m update of W^T with row compaction (out of place): Wt'[i,:] = Wt[si,:] - sum_s U[s,si] C[s,:].
@@ -750,7 +772,7 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
             PhaseScope ps(PH_LAZY_UPDATE_AQ, st);
             {
                 const int T = (n_new + 63) / 64;
-                k_lazy_update_aq<<<dim3(T * (T + 1) / 2, L), 256, 0, st>>>(
+                k_lazy_update_aq<<<dim3(T * (T + 1) / 2, L), 128, 0, st>>>(
                     n_new, nsteps, d, w.A[cur], w.Q[cur], w.A[nxt], w.Q[nxt], w.src, w.U, w.Z);
                 ZIPLM_CHECK_LAUNCH();
             }
