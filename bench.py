@@ -175,8 +175,11 @@ LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in p
 # since the captures.
 NCU_TRAFFIC = {
     # k_lazy_update_aq, first block (n_new = 3040): profiles/k_lazy_kernels_c3_4layers.md
-    "k_lazy_update_aq": dict(bytes=3 * (161.9e6 + 93.5e6), launch="n_new = 3040, m = 32",
+    "k_lazy_update_aq": dict(bytes=3 * (158.6e6 + 89.4e6), launch="n_new = 3040, m = 32",
                              algorithmic=12 * 16.0 * 3040 * 3039 / 2),
+    # k_dgemm_tiles, top-level product F21 = A21 M11^T: profiles/inverse_kernels_c3.md
+    "k_dgemm_tiles": dict(bytes=3 * (114.8e6 + 54.0e6), launch="F21 = A21 M11^T, 24 x 24 tiles",
+                          algorithmic=None),
     # k_neuron_update at n = 3066: profiles/k_neuron_update_c3_4layers.md
     "k_neuron_update": dict(bytes=3 * (113.8e6 + 56.6e6), launch="n = 3066",
                             algorithmic=12 * (8.0 * 768 * 3066 + 4.0 * 3066 * 3066)),
@@ -370,7 +373,9 @@ def run_ours(args, shape):
             gpu_launches=int(launches),
             clocks=clocks,
             roofline=dict(kernel="k_dgemm_tiles", bound="alu", achieved=prod_tflops, peak=fp64_peak,
-                          unit="TFLOP/s", frac=prod_tflops / fp64_peak, traffic=None,
+                          unit="TFLOP/s", frac=prod_tflops / fp64_peak,
+                          traffic=NCU_TRAFFIC["k_dgemm_tiles"]["bytes"] if full_workload else None,
+                          traffic_note=NCU_TRAFFIC["k_dgemm_tiles"],
                           launches=prod_n, avg_launch_us=1e3 * prod_ms / max(prod_n, 1),
                           algorithmic_flop_per_step=prod_flop,
                           peak_source="measured: float64 FMA loop in registers, 36.5 TFLOP/s "
