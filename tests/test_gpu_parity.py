@@ -220,6 +220,38 @@ def test_block_path_with_group_size_one_agrees_with_neuron_path(monkeypatch, neu
         compare_layer(W[l].numpy(), H[l].numpy(), 1, 0.01, [128, 64, 0], b, l)
 
 
+# ------------------------------------------------------------------ exact ties, degenerate shapes
+@pytest.mark.parametrize("g", [1, 4])
+def test_exact_ties_go_to_the_lowest_index(g, neuron_path):
+    """Diagonal H with equal entries and columns of equal norm: every saliency ties exactly, so
+    the removal order must be 0, 1, 2, ... on every path (Eq. 2 gives rho = (h + lambda) ||W_S||^2)."""
+    z = zb()
+    d, r, L = 32, 8, 2
+    H = (3.0 * torch.eye(d))[None].repeat(L, 1, 1).contiguous()
+    W = torch.ones(L, r, d) * 0.5
+    G = d // g
+    out = z.prune_layers(W.cuda(), H.cuda(), g, 0.01, [G // 2, 0])
+    torch.cuda.synchronize()
+    assert out["layer_status"].tolist() == [0] * L
+    for l in range(L):
+        assert out["order"][l].tolist() == list(range(G))
+        compare_layer(W[l].numpy(), H[l].numpy(), g, 0.01, [G // 2, 0], out, l)
+
+
+def test_single_structure_and_no_levels():
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c2_bert_base_attn"][0], d_col=64, d_row=16, group_size=64,
+                   n_tokens=300, n_layers=2, levels=(1, 0))
+    run_case(sh)                                   # G = 1: one step removes the whole module
+    W, X = wl.make_layers(sh, "cpu")
+    H = torch.stack([oracle_h32(X[l]) for l in range(2)])
+    for g in (1, 64):                              # no levels requested: nothing is removed
+        out = z.prune_layers(W.cuda(), H.cuda(), g, 0.01, [])
+        torch.cuda.synchronize()
+        assert out["layer_status"].tolist() == [0, 0]
+        assert torch.all(out["order"] == -1)
+
+
 # ------------------------------------------------------------------ host-side argument checks
 def test_invalid_arguments_are_rejected_on_the_host():
     z = zb()
