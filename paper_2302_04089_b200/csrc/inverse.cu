@@ -24,115 +24,135 @@ static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratch
 
 namespace ziplm {
 namespace {
-constexpr int KC = 8;           // k-chunk staged in shared memory per iteration
-constexpr int LDS = kTile + 2;  // padded shared-memory row length (doubles), keeps rows 16-byte aligned
-constexpr int GT = 64;          // threads of a product CTA: 8 x 8 outputs per thread
+constexpr int KC = 16;          // k-chunk staged in shared memory per pipeline stage
+constexpr int MT = 128;         // edge of the macro tile one CTA computes (2 x 2 tiles)
+constexpr int GT = 512;         // threads of a product CTA: 16 warps, 32 x 32 outputs per warp
+constexpr int kStages = 3;      // cp.async pipeline depth
+// Shared-memory pitches (doubles).  Both are 4 mod 16, so that the 16 threads of a half-warp
+// (4 m-indices x 4 k-indices of an operand fragment) hit 16 different 8-byte banks, and both keep
+// rows 16-byte aligned for cp.async.
+constexpr int P_MK = KC + 4;    // chunk stored [m][k] (k contiguous in global memory)
+constexpr int P_KM = MT + 4;    // chunk stored [k][m] (m contiguous in global memory)
+constexpr int kStageDoubles = MT * P_MK > KC * P_KM ? MT * P_MK : KC * P_KM;
+constexpr size_t kProductSmemBytes = sizeof(double) * 2 * kStages * kStageDoubles;
 
-// Both operands sit in shared memory k-major (s[k][i]): the inner loop then reads two
-// neighbouring rows / columns per 128-bit load, 8 loads for 64 FMAs.
-struct TileSmem {
-    double a[2][KC][LDS];
-    double b[2][KC][LDS];
+__device__ __forceinline__ void cp_async16(double* smem_dst, const double* gmem_src) {
+    const unsigned sa = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// D(8x8) += A(8x4) B(4x8) in float64 on the tensor core.  Lane T holds A[T/4][T%4], B[T%4][T/4]
+// and D[T/4][2(T%4)], D[T/4][2(T%4)+1].
+__device__ __forceinline__ void dmma884(double (&d)[2], double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
+}
+
+// Start the copy of one 128 x KC operand chunk into a pipeline stage; rows m >= m_valid (tiles
+// beyond the edge of the task) are not touched.
+//   KM == false: op(m,k) = P[m*ld + k], kept as s[m][k] (pitch P_MK);
+//   KM == true : op(m,k) = P[k*ld + m], kept as s[k][m] (pitch P_KM).
+template <bool KM>
+__device__ __forceinline__ void chunk_async(double* s, const double* P, int ld, int k0, int m_valid) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int piece = threadIdx.x + e * GT;           // 1024 pieces of 16 bytes
+        if (KM) {
+            const int k = piece >> 6, m = (piece & 63) * 2;
+            if (m < m_valid) cp_async16(s + k * P_KM + m, P + (size_t)(k0 + k) * ld + m);
+        } else {
+            const int m = piece >> 3, k = (piece & 7) * 2;
+            if (m < m_valid) cp_async16(s + m * P_MK + k, P + (size_t)m * ld + k0 + k);
+        }
+    }
+}
+
+// Operand fragment of the k-step kk (4 k's) for the 8 m-indices starting at m0.
+template <bool KM>
+__device__ __forceinline__ double frag(const double* s, int m0, int kk, int lane) {
+    return KM ? s[(kk * 4 + (lane & 3)) * P_KM + m0 + (lane >> 2)]
+              : s[(m0 + (lane >> 2)) * P_MK + kk * 4 + (lane & 3)];
+}
+
+// Accumulators of one warp: 4 x 4 fragments of 8 x 8 = a 32 x 32 block of the macro tile.
+struct WarpAcc {
+    double d[4][4][2];
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) d[i][j][0] = d[i][j][1] = 0.0;
+    }
 };
 
-// Fetch one 64 x KC chunk of an operand into registers (8 doubles per thread) and put it into
-// shared memory as s[k][i].
-//   T == false: stored 64 x K row-major (op(i,k) = P[i*ld + k]): a thread takes one row's 8 k's
-//               and writes them down a column of s (consecutive threads -> consecutive i);
-//   T == true : stored K x 64 (op(i,k) = P[k*ld + i]): a thread takes pairs along i.
-template <bool T>
-__device__ __forceinline__ void chunk_load(double (&r)[8], const double* P, int ld, int k0) {
-    const int tid = threadIdx.x;
-    if (T) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const double2 v = *reinterpret_cast<const double2*>(
-                P + (size_t)(k0 + (tid >> 5) + 2 * e) * ld + (tid & 31) * 2);
-            r[2 * e] = v.x; r[2 * e + 1] = v.y;
-        }
-    } else {
-        const double* src = P + (size_t)tid * ld + k0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const double2 v = *reinterpret_cast<const double2*>(src + 2 * e);
-            r[2 * e] = v.x; r[2 * e + 1] = v.y;
-        }
-    }
-}
-
-template <bool T>
-__device__ __forceinline__ void chunk_store(double (*s)[LDS], const double (&r)[8]) {
-    const int tid = threadIdx.x;
-    if (T) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-            *reinterpret_cast<double2*>(&s[(tid >> 5) + 2 * e][(tid & 31) * 2]) =
-                make_double2(r[2 * e], r[2 * e + 1]);
-    } else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) s[e][tid] = r[e];
-    }
-}
-
-// Row / column of output element (p, q) of thread (ty, tx): pairs of neighbours, 16 apart.
-__device__ __forceinline__ int own_index(int t, int p) { return 2 * t + 16 * (p >> 1) + (p & 1); }
-
-// acc(64x64) += opA(64xK) * opB(Kx64); 64 threads, thread (ty,tx) = (tid/8, tid%8) owns the rows
-// own_index(ty, p) and the columns own_index(tx, q), p, q < 8.  The next chunk is fetched into
-// registers while the current one is multiplied out of shared memory (two buffers, one barrier
-// per chunk).  The operand pointers are deliberately not __restrict__: callers may read tiles
-// written earlier in the same launch sequence.  Ends with __syncthreads().
-//   TA == false: A stored 64 x K row-major; true: stored K x 64.
-//   TB == false: B stored K x 64 row-major; true: stored 64 x K.
+// acc(128x128 macro tile) += opA(128xK) opB(Kx128) over the tile range [kt_lo, kt_hi) of K (in
+// tiles of 64), operands streamed through a three-stage cp.async pipeline with one barrier per
+// chunk.  Warp w owns rows 32 (w / 4) .. and columns 32 (w % 4) .. of the macro tile and only
+// multiplies the chunks of its own range [my_lo, my_hi) (the triangular operands cut the range
+// per 64 x 64 tile; what the other warps' ranges bring into shared memory may be uninitialised
+// and is never read by this warp).  rows_valid / cols_valid crop the macro tile at the edge of
+// the task.  A and B point at k = 0 of the macro tile's rows / columns.
+//   TA == false: A stored m x K row-major; true: stored K x m.
+//   TB == false: B stored K x n row-major; true: stored n x K.
+// The operand pointers are deliberately not __restrict__: callers read tiles written earlier in
+// the same launch sequence.
 template <bool TA, bool TB>
-__device__ __forceinline__ void dgemm_tile(double (&acc)[8][8], const double* A, int lda,
-                                           const double* B, int ldb, int K, TileSmem& sm) {
-    const int tid = threadIdx.x;
-    const int ty = tid >> 3, tx = tid & 7;
-    if (K <= 0) return;
-    constexpr bool LA = TA, LB = !TB;       // loader orientation: true = stored K x 64
-    double ra[8], rb[8];
-    chunk_load<LA>(ra, A, lda, 0);
-    chunk_load<LB>(rb, B, ldb, 0);
-    chunk_store<LA>(sm.a[0], ra);
-    chunk_store<LB>(sm.b[0], rb);
-    __syncthreads();
-    int buf = 0;
-    for (int k0 = 0; k0 < K; k0 += KC) {
-        const bool more = k0 + KC < K;
-        if (more) {
-            chunk_load<LA>(ra, A, lda, k0 + KC);
-            chunk_load<LB>(rb, B, ldb, k0 + KC);
+__device__ __forceinline__ void dgemm_macro(WarpAcc& acc, const double* A, int lda, const double* B,
+                                            int ldb, int kt_lo, int kt_hi, int my_lo, int my_hi,
+                                            int rows_valid, int cols_valid, double* smem) {
+    constexpr bool KA = TA, KB = !TB;       // orientation in memory: true = stored K x m
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int r0 = 32 * (warp >> 2), c0 = 32 * (warp & 3);
+    double* sa = smem;
+    double* sb = smem + kStages * kStageDoubles;
+    const int nchunks = (kt_hi - kt_lo) * (kTile / KC);
+    const int kbase = kt_lo * kTile;
+    for (int c = 0; c < kStages - 1; ++c) {
+        if (c < nchunks) {
+            chunk_async<KA>(sa + c * kStageDoubles, A, lda, kbase + c * KC, rows_valid);
+            chunk_async<KB>(sb + c * kStageDoubles, B, ldb, kbase + c * KC, cols_valid);
         }
+        cp_async_commit();
+    }
+    for (int c = 0; c < nchunks; ++c) {
+        cp_async_wait<kStages - 2>();       // chunk c has landed (this thread's pieces)
+        __syncthreads();                    // ... everyone's; and chunk c - 1 has been consumed
+        const int nx = c + kStages - 1;
+        if (nx < nchunks) {
+            const int st = nx % kStages;
+            chunk_async<KA>(sa + st * kStageDoubles, A, lda, kbase + nx * KC, rows_valid);
+            chunk_async<KB>(sb + st * kStageDoubles, B, ldb, kbase + nx * KC, cols_valid);
+        }
+        cp_async_commit();
+        const int ktile = kt_lo + c / (kTile / KC);
+        if (ktile < my_lo || ktile >= my_hi) continue;
+        const double* pa = sa + (c % kStages) * kStageDoubles;
+        const double* pb = sb + (c % kStages) * kStageDoubles;
 #pragma unroll
-        for (int kk = 0; kk < KC; ++kk) {
-            double a[8], b[8];
+        for (int kk = 0; kk < KC / 4; ++kk) {
+            double a[4], b[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const double2 va = *reinterpret_cast<const double2*>(&sm.a[buf][kk][2 * ty + 16 * q]);
-                const double2 vb = *reinterpret_cast<const double2*>(&sm.b[buf][kk][2 * tx + 16 * q]);
-                a[2 * q] = va.x; a[2 * q + 1] = va.y;
-                b[2 * q] = vb.x; b[2 * q + 1] = vb.y;
+            for (int i = 0; i < 4; ++i) {
+                a[i] = frag<KA>(pa, r0 + 8 * i, kk, lane);
+                b[i] = frag<KB>(pb, c0 + 8 * i, kk, lane);
             }
 #pragma unroll
-            for (int p = 0; p < 8; ++p)
+            for (int i = 0; i < 4; ++i)
 #pragma unroll
-                for (int q = 0; q < 8; ++q) acc[p][q] = fma(a[p], b[q], acc[p][q]);
+                for (int j = 0; j < 4; ++j) dmma884(acc.d[i][j], a[i], b[j]);
         }
-        if (more) {
-            chunk_store<LA>(sm.a[buf ^ 1], ra);
-            chunk_store<LB>(sm.b[buf ^ 1], rb);
-        }
-        __syncthreads();
-        buf ^= 1;
     }
+    cp_async_wait<0>();
 }
 
-__device__ __forceinline__ void zero_acc(double (&acc)[8][8]) {
-#pragma unroll
-    for (int p = 0; p < 8; ++p)
-#pragma unroll
-        for (int q = 0; q < 8; ++q) acc[p][q] = 0.0;
+// Linear index -> (row, col) of the lower triangle, rows in order 0, 1, ...
+__device__ __forceinline__ void lower_index(int idx, int& row, int& col) {
+    row = 0;
+    while (idx > row) { idx -= row + 1; ++row; }
+    col = idx;
 }
 
 // lambda[l] = damp_frac * mean(diag H[l]); flags non-finite diagonals and non-positive means.
@@ -215,38 +235,57 @@ struct GemmTask {
     double alpha; int beta;             // beta in {0, 1}
 };
 
-template <bool TA, bool TB>
-__global__ void __launch_bounds__(GT) k_dgemm_tiles(GemmTask t, int dp) {
-    __shared__ TileSmem sm;
-    const int l = blockIdx.y;
-    int ti, tj;
-    if (t.lower_only) {
-        ti = 0; int rem = blockIdx.x;
-        while (rem > ti) { rem -= ti + 1; ++ti; }
-        tj = rem;
-    } else {
-        ti = blockIdx.x / t.nt; tj = blockIdx.x % t.nt;
-    }
-    int klo = 0, khi = t.kt;
+// k range (in tiles) of output tile (ti, tj) under the task's kmode.
+__device__ __forceinline__ void task_krange(const GemmTask& t, int ti, int tj, int& klo, int& khi) {
+    klo = 0; khi = t.kt;
     if (t.kmode == 1) khi = min(t.kt, tj + 1);
     else if (t.kmode == 2) khi = min(t.kt, ti + 1);
     else if (t.kmode == 3) klo = tj;
+}
+
+// One CTA per 128 x 128 macro tile (2 x 2 tiles); blockIdx.x runs over the macro tiles of the
+// task (the lower triangle of macro tiles when lower_only), blockIdx.y over the layers.
+template <bool TA, bool TB>
+__global__ void __launch_bounds__(GT, 1) k_dgemm_tiles(GemmTask t, int dp) {
+    extern __shared__ __align__(16) double smem[];
+    const int l = blockIdx.y;
+    const int nmt = (t.nt + 1) / 2;
+    int I, J;
+    if (t.lower_only) lower_index(blockIdx.x, I, J);
+    else { I = blockIdx.x / nmt; J = blockIdx.x % nmt; }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ti = 2 * I + (warp >> 3), tj = 2 * J + ((warp >> 1) & 1);   // this warp's tile
+    const bool mine = ti < t.mt && tj < t.nt && (!t.lower_only || ti >= tj);
+    // CTA range: union over its valid tiles; warp range: its own tile's
+    int kt_lo = t.kt, kt_hi = 0;
+    for (int a = 0; a < 2; ++a)
+        for (int b = 0; b < 2; ++b) {
+            const int si = 2 * I + a, sj = 2 * J + b;
+            if (si >= t.mt || sj >= t.nt || (t.lower_only && si < sj)) continue;
+            int lo, hi;
+            task_krange(t, si, sj, lo, hi);
+            kt_lo = min(kt_lo, lo); kt_hi = max(kt_hi, hi);
+        }
+    int my_lo = 0, my_hi = 0;
+    if (mine) task_krange(t, ti, tj, my_lo, my_hi);
+    const int rows_valid = min(MT, (t.mt - 2 * I) * kTile), cols_valid = min(MT, (t.nt - 2 * J) * kTile);
     const size_t lay = (size_t)l * dp * dp;
-    const double* A = t.A + lay + (TA ? ((size_t)(t.a_r + klo) * kTile * dp + (size_t)(t.a_c + ti) * kTile)
-                                      : ((size_t)(t.a_r + ti) * kTile * dp + (size_t)(t.a_c + klo) * kTile));
-    const double* B = t.B + lay + (TB ? ((size_t)(t.b_r + tj) * kTile * dp + (size_t)(t.b_c + klo) * kTile)
-                                      : ((size_t)(t.b_r + klo) * kTile * dp + (size_t)(t.b_c + tj) * kTile));
-    double acc[8][8];
-    zero_acc(acc);
-    dgemm_tile<TA, TB>(acc, A, dp, B, dp, (khi - klo) * kTile, sm);
-    double* out = t.C + lay + (size_t)(t.c_r + ti) * kTile * dp + (size_t)(t.c_c + tj) * kTile;
-    const int ty = threadIdx.x >> 3, tx = threadIdx.x & 7;
+    const double* A = t.A + lay + (TA ? ((size_t)t.a_r * kTile * dp + (size_t)(t.a_c + 2 * I) * kTile)
+                                      : ((size_t)(t.a_r + 2 * I) * kTile * dp + (size_t)t.a_c * kTile));
+    const double* B = t.B + lay + (TB ? ((size_t)(t.b_r + 2 * J) * kTile * dp + (size_t)t.b_c * kTile)
+                                      : ((size_t)t.b_r * kTile * dp + (size_t)(t.b_c + 2 * J) * kTile));
+    WarpAcc acc;
+    acc.zero();
+    dgemm_macro<TA, TB>(acc, A, dp, B, dp, kt_lo, kt_hi, my_lo, my_hi, rows_valid, cols_valid, smem);
+    if (!mine) return;
+    double* out = t.C + lay + (size_t)((t.c_r + 2 * I) * kTile + 32 * (warp >> 2)) * dp +
+                  (size_t)(t.c_c + 2 * J) * kTile + 32 * (warp & 3);
 #pragma unroll
-    for (int p = 0; p < 8; ++p)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int q = 0; q < 8; q += 2) {
-            double2* o = reinterpret_cast<double2*>(out + (size_t)own_index(ty, p) * dp + own_index(tx, q));
-            double2 v = make_double2(t.alpha * acc[p][q], t.alpha * acc[p][q + 1]);
+        for (int j = 0; j < 4; ++j) {
+            double2* o = reinterpret_cast<double2*>(out + (size_t)(8 * i + (lane >> 2)) * dp + 8 * j + 2 * (lane & 3));
+            double2 v = make_double2(t.alpha * acc.d[i][j][0], t.alpha * acc.d[i][j][1]);
             if (t.beta) { const double2 c = *o; v.x += c.x; v.y += c.y; }
             *o = v;
         }
@@ -323,36 +362,44 @@ __global__ void __launch_bounds__(256) k_potf2(const double* A, double* F, doubl
 
 // H^-1 = M^T M on the lower tiles (i >= j): sum over k >= i of M_ki^T M_kj; writes the cropped
 // d x d result as float64 (mirrored to the upper triangle) and/or fp32 strict lower + fp64 diag.
-__global__ void __launch_bounds__(GT) k_lauum(const double* M, int dp, int T, int d, double* out64,
-                                              float* tri32, int pitch32, double* diag64) {
-    __shared__ TileSmem sm;
+// One CTA per 128 x 128 macro tile of the lower triangle.
+__global__ void __launch_bounds__(GT, 1) k_lauum(const double* M, int dp, int T, int d, double* out64,
+                                                 float* tri32, int pitch32, double* diag64) {
+    extern __shared__ __align__(16) double smem[];
     const int l = blockIdx.y;
-    // linear tile index -> (i, j), rows of the lower triangle in order i = 0, 1, ...
-    int i = 0, rem = blockIdx.x;
-    while (rem > i) { rem -= i + 1; ++i; }
-    const int j = rem;
+    int I, J;
+    lower_index(blockIdx.x, I, J);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ti = 2 * I + (warp >> 3), tj = 2 * J + ((warp >> 1) & 1);
+    const bool mine = ti < T && tj < T && ti >= tj;
     const double* Ml = M + (size_t)l * dp * dp;
-    double acc[8][8];
-    zero_acc(acc);
-    dgemm_tile<true, false>(acc, Ml + (size_t)i * kTile * dp + (size_t)i * kTile, dp,
-                            Ml + (size_t)i * kTile * dp + (size_t)j * kTile, dp, (T - i) * kTile, sm);
-    const int ty = threadIdx.x >> 3, tx = threadIdx.x & 7;
+    const int rows_valid = min(MT, (T - 2 * I) * kTile), cols_valid = min(MT, (T - 2 * J) * kTile);
+    WarpAcc acc;
+    acc.zero();
+    // (M^T M)_ij: opA(i,k) = M[k][i] (stored K x m), opB(k,j) = M[k][j]; tile (ti, .) starts at k = ti
+    dgemm_macro<true, false>(acc, Ml + (size_t)(2 * I) * kTile, dp, Ml + (size_t)(2 * J) * kTile, dp,
+                             2 * I, T, mine ? ti : 0, mine ? T : 0, rows_valid, cols_valid, smem);
+    if (!mine) return;
+    const int row0 = 2 * I * kTile + 32 * (warp >> 2) + (lane >> 2);
+    const int col0 = 2 * J * kTile + 32 * (warp & 3) + 2 * (lane & 3);
 #pragma unroll
-    for (int p = 0; p < 8; ++p)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int row = i * kTile + own_index(ty, p), col = j * kTile + own_index(tx, q);
-            if (row >= d || col >= d) continue;
-            const double v = acc[p][q];
-            if (out64 && row >= col) {
-                double* o = out64 + (size_t)l * d * d;
-                o[(size_t)row * d + col] = v;
-                o[(size_t)col * d + row] = v;
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int row = row0 + 8 * i, col = col0 + 8 * j + e;
+                if (row >= d || col >= d) continue;
+                const double v = acc.d[i][j][e];
+                if (out64 && row >= col) {
+                    double* o = out64 + (size_t)l * d * d;
+                    o[(size_t)row * d + col] = v;
+                    o[(size_t)col * d + row] = v;
+                }
+                if (tri32 && row > col)
+                    tri32[(size_t)l * d * pitch32 + (size_t)row * pitch32 + col] = (float)v;
+                if (diag64 && row == col) diag64[(size_t)l * d + row] = v;
             }
-            if (tri32 && row > col)
-                tri32[(size_t)l * d * pitch32 + (size_t)row * pitch32 + col] = (float)v;
-            if (diag64 && row == col) diag64[(size_t)l * d + row] = v;
-        }
 }
 
 struct InvCtx {
@@ -366,10 +413,14 @@ struct InvCtx {
 
 template <bool TA, bool TB>
 ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
-    const int tiles = t.lower_only ? t.mt * (t.mt + 1) / 2 : t.mt * t.nt;
-    if (tiles <= 0 || t.kt <= 0) return ZIPLM_OK;
+    const int mm = (t.mt + 1) / 2, nm = (t.nt + 1) / 2;      // macro tiles
+    const int ctas = t.lower_only ? mm * (mm + 1) / 2 : mm * nm;
+    if (ctas <= 0 || t.kt <= 0) return ZIPLM_OK;
+    static const cudaError_t attr = cudaFuncSetAttribute(
+        k_dgemm_tiles<TA, TB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
+    if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
     PhaseScope ps(PH_INV_PRODUCTS, c.st);
-    k_dgemm_tiles<TA, TB><<<dim3(tiles, c.L), GT, 0, c.st>>>(t, c.dp);
+    k_dgemm_tiles<TA, TB><<<dim3(ctas, c.L), GT, kProductSmemBytes, c.st>>>(t, c.dp);
     ZIPLM_CHECK_LAUNCH();
     return ZIPLM_OK;
 }
@@ -436,7 +487,12 @@ ziplm_status run_damped_inverse(const float* H, int L, int d, float damp_frac, d
     if (s != ZIPLM_OK) return s;
     {
         PhaseScope ps(PH_INV_LAUUM, st);
-        k_lauum<<<dim3(T * (T + 1) / 2, L), GT, 0, st>>>(ctx.M, dp, T, d, out64, tri32, pitch32, diag64);
+        static const cudaError_t attr = cudaFuncSetAttribute(
+            k_lauum, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
+        if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
+        const int Tm = (T + 1) / 2;
+        k_lauum<<<dim3(Tm * (Tm + 1) / 2, L), GT, kProductSmemBytes, st>>>(ctx.M, dp, T, d, out64, tri32,
+                                                                         pitch32, diag64);
         ZIPLM_CHECK_LAUNCH();
     }
     if (lam_out) {
