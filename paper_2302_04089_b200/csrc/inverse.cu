@@ -249,9 +249,13 @@ template <bool TA, bool TB>
 __global__ void __launch_bounds__(GT, 1) k_dgemm_tiles(GemmTask t, int dp) {
     extern __shared__ __align__(16) double smem[];
     const int l = blockIdx.y;
-    const int nmt = (t.nt + 1) / 2;
+    const int mmt = (t.mt + 1) / 2, nmt = (t.nt + 1) / 2;
+    // macro tiles with the longest k range come first, so that the last wave is the lightest
     int I, J;
     if (t.lower_only) lower_index(blockIdx.x, I, J);
+    else if (t.kmode == 1) { J = nmt - 1 - blockIdx.x / mmt; I = blockIdx.x % mmt; }
+    else if (t.kmode == 3) { J = blockIdx.x / mmt; I = blockIdx.x % mmt; }
+    else if (t.kmode == 2) { I = mmt - 1 - blockIdx.x / nmt; J = blockIdx.x % nmt; }
     else { I = blockIdx.x / nmt; J = blockIdx.x % nmt; }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ti = 2 * I + (warp >> 3), tj = 2 * J + ((warp >> 1) & 1);   // this warp's tile
@@ -291,73 +295,336 @@ __global__ void __launch_bounds__(GT, 1) k_dgemm_tiles(GemmTask t, int dp) {
         }
 }
 
-// Leaf of the recursion: unblocked Cholesky of the diagonal tile A_jj -> F_jj (lower, upper part
-// zeroed) and the inverse of that factor -> M_jj (lower, upper part zeroed).
-__global__ void __launch_bounds__(256) k_potf2(const double* A, double* F, double* M, int dp, int j,
-                                               int* layer_status) {
-    __shared__ double s[kTile][kTile + 1];
-    __shared__ double dinv[kTile];
-    __shared__ int sflag;
-    const int l = blockIdx.x;
-    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-    const size_t off = (size_t)l * dp * dp + (size_t)j * kTile * dp + (size_t)j * kTile;
-    if (tid == 0) sflag = 0;
-    for (int e = tid; e < kTile * kTile; e += 256)
-        s[e >> 6][e & 63] = A[off + (size_t)(e >> 6) * dp + (e & 63)];
+// ---- base case of the recursion: a range of up to kSmallMax tiles, one CTA per layer ----------
+constexpr int kSmallMax = 4;
+constexpr int PS = kTile + 4;    // pitch of a 64 x 64 operand tile in shared memory (4 mod 16)
+
+struct SmallSmem {
+    double ta[kTile * PS];       // operand tiles, as stored (row-major)
+    double tb[kTile * PS];
+    double td[kTile * PS];       // inverse of the current diagonal factor tile
+    double s[kTile][kTile + 1];  // leaf work array: the factor (lower part)
+    double col[2][kTile];        // current column of the leaf factorisation (double-buffered)
+    double dinv[kTile];          // reciprocal diagonal of the factor
+    int flag;                    // first error seen by this CTA
+};
+
+// Start the copy of a 64 x 64 tile (row-major, leading dimension ld) into a shared-memory tile.
+__device__ __forceinline__ void tile_async(double* dst, const double* src, int ld) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int piece = threadIdx.x + e * GT;            // 2048 pieces of 16 bytes
+        const int r = piece >> 5, c = (piece & 31) * 2;
+        cp_async16(dst + r * PS + c, src + (size_t)r * ld + c);
+    }
+}
+
+// Fragment of a shared-memory tile: KM == false: op(m,k) = s[m][k]; true: op(m,k) = s[k][m].
+template <bool KM>
+__device__ __forceinline__ double tile_frag(const double* s, int m0, int kk, int lane) {
+    return KM ? s[(kk * 4 + (lane & 3)) * PS + m0 + (lane >> 2)]
+              : s[(m0 + (lane >> 2)) * PS + kk * 4 + (lane & 3)];
+}
+
+// Accumulators of one warp of the small kernel: 2 x 2 fragments = a 16 x 16 block of a tile;
+// warp w owns rows 16 (w / 4) .. and columns 16 (w % 4) ...
+struct SmallAcc {
+    double d[2][2][2];
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) d[i][j][0] = d[i][j][1] = 0.0;
+    }
+};
+
+// acc += opA(64 x 64) opB(64 x 64), both operands in shared memory.
+//   AKM: opA(m,k) = sa[k][m], else sa[m][k];  BKN: opB(k,n) = sb[k][n], else sb[n][k].
+template <bool AKM, bool BKN>
+__device__ __forceinline__ void tile_mma(SmallAcc& acc, const double* sa, const double* sb) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int r0 = 16 * (warp >> 2), c0 = 16 * (warp & 3);
+#pragma unroll 4
+    for (int kk = 0; kk < kTile / 4; ++kk) {
+        double a[2], b[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            a[i] = tile_frag<AKM>(sa, r0 + 8 * i, kk, lane);
+            b[i] = tile_frag<BKN>(sb, c0 + 8 * i, kk, lane);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) dmma884(acc.d[i][j], a[i], b[j]);
+    }
+}
+
+// Visit the elements of a warp's accumulators: f(row, col, pair) with col even.
+template <typename Fn>
+__device__ __forceinline__ void small_epilogue(const SmallAcc& acc, Fn f) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int r0 = 16 * (warp >> 2) + (lane >> 2), c0 = 16 * (warp & 3) + 2 * (lane & 3);
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            f(r0 + 8 * i, c0 + 8 * j, make_double2(acc.d[i][j][0], acc.d[i][j][1]));
+}
+
+// One warp: acc(16 x 16) += A(16 x K) B(K x 16), operands anywhere in shared memory
+// (A[m * lda + k], B[k * ldb + n]); K a multiple of 4.
+__device__ __forceinline__ void warp_mma16(double (&acc)[2][2][2], const double* A, int lda,
+                                           const double* B, int ldb, int K) {
+    const int lane = threadIdx.x & 31;
+    for (int k0 = 0; k0 < K; k0 += 4) {
+        double a[2], b[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            a[i] = A[(8 * i + (lane >> 2)) * lda + k0 + (lane & 3)];
+            b[i] = B[(k0 + (lane & 3)) * ldb + 8 * i + (lane >> 2)];
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) dmma884(acc[i][j], a[i], b[j]);
+    }
+}
+
+// One warp: C(16 x 16) = sign * acc, C[m * ldc + n].
+__device__ __forceinline__ void warp_store16(const double (&acc)[2][2][2], double* C, int ldc, double sign) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+                C[(8 * i + (lane >> 2)) * ldc + 8 * j + 2 * (lane & 3) + e] = sign * acc[i][j][e];
+}
+
+// Leaf: Cholesky factor of the 64 x 64 tile at Ag -> Fg (lower, upper part zeroed), the inverse of
+// that factor -> Mg and sm.td (lower, upper part zeroed).  Starts and ends with a barrier.
+//   Factor: threads 0..255 hold the tile in registers, cyclically (rows ty + 16 a, columns
+//   tx + 16 b, tx constant over half a warp), so a column step is one barrier, eight
+//   shared-memory reads and 16 FMAs per thread; only the warp that owns the column publishes it.
+//   Inverse: the four 16 x 16 diagonal blocks by forward substitution (one thread per column),
+//   then the off-diagonal blocks of the 32- and 64-wide levels as products
+//   M21 = -M22 (L21 M11) on the tensor core.
+__device__ __forceinline__ void leaf_factor(const double* Ag, double* Fg, double* Mg, int dp,
+                                            SmallSmem& sm) {
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const bool worker = tid < 256;
+    const int ty = tid & 15, tx = (tid >> 4) & 15;
+    __syncthreads();                          // earlier readers of the shared arrays are done
+    tile_async(sm.tb, Ag, dp);
+    cp_async_commit();
+    for (int e = tid; e < kTile * PS; e += GT) sm.ta[e] = 0.0;   // the inverse is built in ta
+    cp_async_wait<0>();
     __syncthreads();
+    double r[4][4];
+    if (worker) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) r[a][b] = sm.tb[(ty + 16 * a) * PS + tx + 16 * b];
+    }
     for (int c = 0; c < kTile; ++c) {
-        // every thread forms 1/sqrt(pivot) itself: no broadcast, two barriers per column
-        double p = s[c][c];
-        if (!(p > 0.0) || !isfinite(p)) {   // not positive definite (or NaN): flag, keep going
-            if (tid == 0 && !sflag) sflag = isfinite(p) ? ZIPLM_ERR_NOT_PD : ZIPLM_ERR_NONFINITE;
-            p = 1.0;
-        }
-        const double rinv = rsqrt(p);
-        __syncthreads();                    // all threads have read the pivot
-        if (tid == c) s[c][c] = p * rinv;
-        else if (tid > c && tid < kTile) s[tid][c] *= rinv;
-        __syncthreads();
-        // trailing update of the lower triangle: rows ty + 16a, cols tx + 16b
+        const int cb = c >> 4, ct = c & 15;
+        double* col = sm.col[c & 1];
+        if (worker && tx == ct) {
 #pragma unroll
-        for (int a = 0; a < 4; ++a) {
-            const int i = ty + 16 * a;
-            if (i <= c) continue;
-            const double lic = s[i][c];
+            for (int a = 0; a < 4; ++a) {
+                double v = r[a][0];
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const int jj = tx + 16 * b;
-                if (jj > c && jj <= i) s[i][jj] -= lic * s[jj][c];
+                for (int b = 1; b < 4; ++b) v = (b == cb) ? r[a][b] : v;
+                col[ty + 16 * a] = v;
             }
         }
         __syncthreads();
+        if (worker) {
+            double p = col[c];
+            if (!(p > 0.0) || !isfinite(p)) {   // not positive definite (or NaN): flag, keep going
+                if (tid == 0 && !sm.flag) sm.flag = isfinite(p) ? ZIPLM_ERR_NOT_PD : ZIPLM_ERR_NONFINITE;
+                p = 1.0;
+            }
+            const double rinv = rsqrt(p);
+            if (tid == 0) sm.dinv[c] = rinv;    // 1 / L_cc
+            double li[4], lj[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                li[a] = col[ty + 16 * a] * rinv;
+                lj[a] = col[tx + 16 * a] * rinv;
+            }
+            // Columns <= c are final.  Rows <= c of the later columns lie above the diagonal:
+            // they are never used, so they are updated along with the rest.
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                if (tx + 16 * b > c) {
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) r[a][b] = fma(-li[a], lj[b], r[a][b]);
+                }
+            if (tx == ct) {
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+                    const int i = ty + 16 * a;
+                    const double v = i > c ? li[a] : p * rinv;
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+                        if (b == cb && i >= c) r[a][b] = v;
+                }
+            }
+        }
     }
-    // inverse of the lower-triangular factor: thread `cidx` builds column cidx by forward
-    // substitution.  Entry (i, cidx), i > cidx, is parked transposed in the unused strict upper
-    // triangle of s (slot [cidx][i]); the reciprocal diagonal goes to dinv first.
-    if (tid < kTile) dinv[tid] = 1.0 / s[tid][tid];
+    if (worker) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                if (tx + 16 * b <= ty + 16 * a) sm.s[ty + 16 * a][tx + 16 * b] = r[a][b];
+    }
     __syncthreads();
+    // ---- inverse of the factor, built in sm.ta (pitch PS, zero above the diagonal) ----
     if (tid < kTile) {
-        const int cidx = tid;
-        for (int i = cidx + 1; i < kTile; ++i) {
-            double a0 = -s[i][cidx] * dinv[cidx], a1 = 0.0, a2 = 0.0, a3 = 0.0;
-            int k = cidx + 1;
-            for (; k + 3 < i; k += 4) {
-                a0 = fma(-s[i][k], s[cidx][k], a0);
-                a1 = fma(-s[i][k + 1], s[cidx][k + 1], a1);
-                a2 = fma(-s[i][k + 2], s[cidx][k + 2], a2);
-                a3 = fma(-s[i][k + 3], s[cidx][k + 3], a3);
-            }
-            for (; k < i; ++k) a0 = fma(-s[i][k], s[cidx][k], a0);
-            s[cidx][i] = ((a0 + a1) + (a2 + a3)) * dinv[i];
+        // column cc of diagonal block q: x_i = (delta_i,cc - sum_{cc <= k < i} L_ik x_k) / L_ii
+        const int q0 = tid & ~15, cc = tid & 15;
+        double x[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            double acc = (i == cc) ? 1.0 : 0.0;
+#pragma unroll
+            for (int k = 0; k < i; ++k) acc = fma(-sm.s[q0 + i][q0 + k], x[k], acc);
+            x[i] = (i >= cc) ? acc * sm.dinv[q0 + i] : 0.0;
+            sm.ta[(q0 + i) * PS + q0 + cc] = x[i];
         }
     }
     __syncthreads();
-    for (int e = tid; e < kTile * kTile; e += 256) {
-        const int i = e >> 6, jj = e & 63;
-        F[off + (size_t)i * dp + jj] = (jj <= i) ? s[i][jj] : 0.0;
-        M[off + (size_t)i * dp + jj] = (jj < i) ? s[jj][i] : (jj == i ? dinv[i] : 0.0);
+    double acc[2][2][2];
+    auto zero = [&]() {
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+    };
+    // 32-wide level: blocks (1,0) and (3,2) of 16 x 16; warp q does pair q.  tb holds L21 M11.
+    if (warp < 2) {
+        const int o = 32 * warp;
+        zero();
+        warp_mma16(acc, &sm.s[o + 16][o], kTile + 1, sm.ta + o * PS + o, PS, 16);
+        warp_store16(acc, sm.tb + (o + 16) * PS + o, PS, 1.0);
     }
-    if (tid == 0 && sflag) set_layer_status(layer_status, l, sflag);
+    __syncthreads();
+    if (warp < 2) {
+        const int o = 32 * warp;
+        zero();
+        warp_mma16(acc, sm.ta + (o + 16) * PS + o + 16, PS, sm.tb + (o + 16) * PS + o, PS, 16);
+        warp_store16(acc, sm.ta + (o + 16) * PS + o, PS, -1.0);
+    }
+    __syncthreads();
+    // 64-wide level: block (rows 32.., cols 0..31); warp w < 4 does the 16 x 16 part (w / 2, w % 2).
+    if (warp < 4) {
+        const int rb = 32 + 16 * (warp >> 1), cb = 16 * (warp & 1);
+        zero();
+        warp_mma16(acc, &sm.s[rb][0], kTile + 1, sm.ta + cb, PS, 32);
+        warp_store16(acc, sm.tb + rb * PS + cb, PS, 1.0);
+    }
+    __syncthreads();
+    if (warp < 4) {
+        const int rb = 32 + 16 * (warp >> 1), cb = 16 * (warp & 1);
+        zero();
+        warp_mma16(acc, sm.ta + rb * PS + 32, PS, sm.tb + 32 * PS + cb, PS, 32);
+        warp_store16(acc, sm.ta + rb * PS + cb, PS, -1.0);
+    }
+    __syncthreads();
+    for (int e = tid; e < kTile * kTile; e += GT) {
+        const int i = e >> 6, jj = e & 63;
+        const double m = sm.ta[i * PS + jj];
+        Fg[(size_t)i * dp + jj] = (jj <= i) ? sm.s[i][jj] : 0.0;
+        Mg[(size_t)i * dp + jj] = m;
+        sm.td[i * PS + jj] = m;
+    }
+    __syncthreads();
+}
+
+// Factor the tile range [lo, lo + nt), nt <= kSmallMax, of every layer with one CTA per layer:
+// right-looking tile Cholesky (A -> F) followed by the block forward substitution for M = F^-1.
+// Every product is a 64 x 64 x 64 tile product of the whole CTA on the float64 tensor core, with
+// its operands fetched from global memory (the L2) into shared memory.
+__global__ void __launch_bounds__(GT, 1) k_factor_small(double* A, double* F, double* M, int dp, int lo,
+                                                        int nt, int* layer_status) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SmallSmem& sm = *reinterpret_cast<SmallSmem*>(smem_raw);
+    const int l = blockIdx.x;
+    const size_t lay = (size_t)l * dp * dp;
+    auto tile = [&](double* base, int i, int j) {
+        return base + lay + (size_t)(lo + i) * kTile * dp + (size_t)(lo + j) * kTile;
+    };
+    if (threadIdx.x == 0) sm.flag = 0;
+    SmallAcc acc;
+    for (int j = 0; j < nt; ++j) {
+        leaf_factor(tile(A, j, j), tile(F, j, j), tile(M, j, j), dp, sm);
+        // F_ij = A_ij D_j^T
+        for (int i = j + 1; i < nt; ++i) {
+            tile_async(sm.ta, tile(A, i, j), dp);
+            cp_async_commit();
+            cp_async_wait<0>();
+            __syncthreads();
+            acc.zero();
+            tile_mma<false, false>(acc, sm.ta, sm.td);
+            double* out = tile(F, i, j);
+            small_epilogue(acc, [&](int r, int c, double2 v) {
+                *reinterpret_cast<double2*>(out + (size_t)r * dp + c) = v;
+            });
+            __syncthreads();
+        }
+        // A_ik -= F_ij F_kj^T for j < k <= i
+        for (int i = j + 1; i < nt; ++i)
+            for (int k = j + 1; k <= i; ++k) {
+                tile_async(sm.ta, tile(F, i, j), dp);
+                tile_async(sm.tb, tile(F, k, j), dp);
+                cp_async_commit();
+                cp_async_wait<0>();
+                __syncthreads();
+                acc.zero();
+                tile_mma<false, false>(acc, sm.ta, sm.tb);
+                double* out = tile(A, i, k);
+                small_epilogue(acc, [&](int r, int c, double2 v) {
+                    double2* o = reinterpret_cast<double2*>(out + (size_t)r * dp + c);
+                    double2 cur = *o;
+                    cur.x -= v.x; cur.y -= v.y;
+                    *o = cur;
+                });
+                __syncthreads();
+            }
+    }
+    // M_ij = -M_ii (sum over j <= k < i of F_ik M_kj), column by column
+    for (int j = 0; j < nt; ++j)
+        for (int i = j + 1; i < nt; ++i) {
+            acc.zero();
+            for (int k = j; k < i; ++k) {
+                tile_async(sm.ta, tile(F, i, k), dp);
+                tile_async(sm.tb, tile(M, k, j), dp);
+                cp_async_commit();
+                cp_async_wait<0>();
+                __syncthreads();
+                tile_mma<false, true>(acc, sm.ta, sm.tb);
+                __syncthreads();
+            }
+            tile_async(sm.ta, tile(M, i, i), dp);
+            cp_async_commit();
+            small_epilogue(acc, [&](int r, int c, double2 v) {
+                *reinterpret_cast<double2*>(sm.tb + r * PS + c) = v;
+            });
+            cp_async_wait<0>();
+            __syncthreads();
+            acc.zero();
+            tile_mma<false, true>(acc, sm.ta, sm.tb);
+            double* out = tile(M, i, j);
+            small_epilogue(acc, [&](int r, int c, double2 v) {
+                *reinterpret_cast<double2*>(out + (size_t)r * dp + c) = make_double2(-v.x, -v.y);
+            });
+            __syncthreads();
+        }
+    if (threadIdx.x == 0 && sm.flag) set_layer_status(layer_status, l, sm.flag);
 }
 
 // H^-1 = M^T M on the lower tiles (i >= j): sum over k >= i of M_ki^T M_kj; writes the cropped
@@ -428,9 +695,13 @@ ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
 // Factor the tile range [lo, hi): on return F holds the Cholesky factor of the (updated) block
 // and M its inverse.
 ziplm_status factor_range(const InvCtx& c, int lo, int hi) {
-    if (hi - lo == 1) {
+    if (hi - lo <= kSmallMax) {
+        static const cudaError_t attr = cudaFuncSetAttribute(
+            k_factor_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmallSmem));
+        if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
         PhaseScope ps(PH_INV_LEAVES, c.st);
-        k_potf2<<<c.L, 256, 0, c.st>>>(c.A, c.F, c.M, c.dp, lo, c.layer_status);
+        k_factor_small<<<c.L, GT, sizeof(SmallSmem), c.st>>>(c.A, c.F, c.M, c.dp, lo, hi - lo,
+                                                              c.layer_status);
         ZIPLM_CHECK_LAUNCH();
         return ZIPLM_OK;
     }
