@@ -380,6 +380,19 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
     cluster.sync();      // no CTA may retire while another can still read its shared memory
 }
 
+// 4-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros without reading.
+__device__ __forceinline__ void cp_async4(float* smem_dst, const float* gmem_src, unsigned src_bytes) {
+    const unsigned sa = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(sa), "l"(gmem_src), "r"(src_bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void cp_async16_zfill(float4* smem_dst, const float* gmem_src, unsigned src_bytes) {
+    const unsigned sa = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(sa), "l"(gmem_src), "r"(src_bytes)
+                 : "memory");
+}
+
 // Rank-m update of the strict lower triangles of H^-1 and Q with compaction (out of place):
 //   A'[i,j] = A[si,sj] - sum_s U[s,si] U[s,sj],
 //   Q'[i,j] = Q[si,sj] - sum_s (Z[s,si] U[s,sj] + U[s,si] Z[s,sj]),    si = src[i] > sj = src[j].
@@ -408,6 +421,9 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
     if (tid < 64) srow[tid] = (i0 + tid < n_new) ? sl[i0 + tid] : -1;
     else scol[tid - 64] = (j0 + tid - 64 < n_new) ? sl[j0 + tid - 64] : -1;
     __syncthreads();
+    // The pending slabs of the tile's rows and columns go straight to shared memory with
+    // asynchronous 4-byte copies (zero-filled past the last live row), so that all of them and the
+    // gathered old entries below are in flight together.
     const float* Ul = U + (size_t)l * BMAX * d;
     const float* Zl = Z + (size_t)l * BMAX * d;
     {
@@ -415,11 +431,13 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
         const int idx = (tid < 64) ? srow[c] : scol[c];
         float (*dU)[64] = (tid < 64) ? sUr : sUc;
         float (*dZ)[64] = (tid < 64) ? sZr : sZc;
-#pragma unroll 4
+        const unsigned nbytes = idx >= 0 ? 4u : 0u;
+        const size_t off = idx >= 0 ? (size_t)idx : 0;
         for (int s = 0; s < m; ++s) {
-            dU[s][c] = idx >= 0 ? Ul[(size_t)s * d + idx] : 0.f;
-            dZ[s][c] = idx >= 0 ? Zl[(size_t)s * d + idx] : 0.f;
+            cp_async4(&dU[s][c], Ul + (size_t)s * d + off, nbytes);
+            cp_async4(&dZ[s][c], Zl + (size_t)s * d + off, nbytes);
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
     }
     const float* Al = A + (size_t)l * d * d;
     const float* Ql = Q + (size_t)l * d * d;
@@ -443,6 +461,7 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
             }
         }
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     for (int s = 0; s < m; ++s) {
         float ur[8], zr[8];
@@ -501,14 +520,16 @@ __global__ void __launch_bounds__(256) k_lazy_update_w(int n_new, int m, int d, 
     __syncthreads();
     const float* Ul = U + (size_t)l * BMAX * d;
     const float* Cl = C + (size_t)l * BMAX * rp;
+    // asynchronous copies (zero-filled where there is nothing to read), in flight together with
+    // the gathered rows below
     for (int e = tid; e < m * 64; e += 256) {
         const int s = e >> 6, c = e & 63;
         const int sr = srow[c];
-        sUr[s][c] = sr >= 0 ? Ul[(size_t)s * d + sr] : 0.f;
+        cp_async4(&sUr[s][c], Ul + (size_t)s * d + (sr >= 0 ? sr : 0), sr >= 0 ? 4u : 0u);
         const int col = c0 + 4 * c;
-        sC[s][c] = (col < rp) ? *reinterpret_cast<const float4*>(Cl + (size_t)s * rp + col)
-                              : make_float4(0.f, 0.f, 0.f, 0.f);
+        cp_async16_zfill(&sC[s][c], Cl + (size_t)s * rp + (col < rp ? col : 0), col < rp ? 16u : 0u);
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
     const int col = c0 + 4 * tx;
     const bool col_ok = col < rp;
     float4 w[16];
@@ -519,6 +540,7 @@ __global__ void __launch_bounds__(256) k_lazy_update_w(int n_new, int m, int d, 
                    ? __ldcs(reinterpret_cast<const float4*>(Wt + (size_t)l * d * rp + (size_t)sr * rp + col))
                    : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     for (int s = 0; s < m; ++s) {
         const float4 c = sC[s][tx];
