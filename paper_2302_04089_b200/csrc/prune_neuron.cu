@@ -388,10 +388,11 @@ static bool use_lazy_path(int d) {
 // few dozen SMs, the panel steps of the factorisation even fewer).  Layers are independent, so
 // they are split into groups that run the whole pipeline on streams of their own: one group's
 // latency-bound kernels then overlap the other groups' bandwidth- and ALU-bound ones.
-constexpr int kMaxGroups = 4;
+constexpr int kMaxGroups = 8;
+constexpr int kDefaultGroups = 4;
 
 static int layer_groups(int L) {
-    int g = kMaxGroups;
+    int g = kDefaultGroups;
     const char* e = getenv("ZIPLM_LAYER_GROUPS");
     if (e) g = atoi(e);
     if (g < 1) g = 1;
