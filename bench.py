@@ -175,10 +175,10 @@ LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in p
 # since the captures.
 NCU_TRAFFIC = {
     # k_lazy_update_aq, first block (n_new = 3040): profiles/k_lazy_kernels_c3_4layers.md
-    "k_lazy_update_aq": dict(bytes=3 * (158.6e6 + 89.4e6), launch="n_new = 3040, m = 32",
+    "k_lazy_update_aq": dict(bytes=3 * (164.0e6 + 90.1e6), launch="n_new = 3040, m = 32",
                              algorithmic=12 * 16.0 * 3040 * 3039 / 2),
     # k_dgemm_tiles, top-level product F21 = A21 M11^T: profiles/inverse_kernels_c3.md
-    "k_dgemm_tiles": dict(bytes=3 * (114.8e6 + 54.0e6), launch="F21 = A21 M11^T, 24 x 24 tiles",
+    "k_dgemm_tiles": dict(bytes=3 * (116.7e6 + 47.3e6), launch="F21 = A21 M11^T, 12 x 12 macro tiles",
                           algorithmic=None),
     # k_neuron_update at n = 3066: profiles/k_neuron_update_c3_4layers.md
     "k_neuron_update": dict(bytes=3 * (113.8e6 + 56.6e6), launch="n = 3066",
@@ -349,7 +349,7 @@ def run_ours(args, shape):
         prod_ms, prod_n = phases.get("inverse_products", (0.0, 0))
         prod_flop = L * (2.0 / 3.0) * float(d) ** 3
         prod_tflops = prod_flop / (prod_ms * 1e-3) / 1e12 if prod_ms > 0 else 0.0
-        fp64_peak = 36.5                                # TFLOP/s, measured with a register-only FMA loop
+        fp64_peak = 37.0      # TFLOP/s, measured with a register-only loop of the float64 mma instruction
         aq_ms, aq_n = phases.get("lazy_update_aq", (0.0, 0))
         aq_bytes, aq_fma, _ = lazy_update_work(L, G, levels)
         aq_gbs = aq_bytes / (aq_ms * 1e-3) / 1e9 if aq_ms > 0 else 0.0
@@ -378,8 +378,9 @@ def run_ours(args, shape):
                           traffic_note=NCU_TRAFFIC["k_dgemm_tiles"],
                           launches=prod_n, avg_launch_us=1e3 * prod_ms / max(prod_n, 1),
                           algorithmic_flop_per_step=prod_flop,
-                          peak_source="measured: float64 FMA loop in registers, 36.5 TFLOP/s "
-                                      "(nominal 148 SMs x 64 lanes x 2 x 1.965 GHz = 37.2)",
+                          peak_source="measured: register-only loop of mma.sync.m8n8k4.f64, 37.0 TFLOP/s "
+                                      "(plain FMA loop 36.5; nominal 148 SMs x 64 lanes x 2 x 1.965 GHz "
+                                      "= 37.2)",
                           note="float64 tile products of the Cholesky factor and its inverse "
                                "(2/3 d^3 flop per layer), the largest share of the step"),
             roofline_lazy_update=dict(kernel="k_lazy_update_aq", bound="hbm", achieved=aq_gbs, peak=peak,

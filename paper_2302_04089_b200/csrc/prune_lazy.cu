@@ -515,7 +515,8 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
 
 // Rank-m update of W^T with row compaction (out of place): Wt'[i,:] = Wt[si,:] - sum_s U[s,si] C[s,:].
 // A CTA owns 64 rows x 256 columns; the C panel and the rows' U entries are staged in shared
-// memory once per CTA, each thread carries 16 rows of one float4 column.
+// memory once per CTA, each thread carries 16 consecutive rows of one float4 column (per pending
+// step: one 128-bit load of C and four broadcast 128-bit loads of U for 64 FMAs).
 __global__ void __launch_bounds__(256) k_lazy_update_w(int n_new, int m, int d, int rp,
                                                        const float* __restrict__ Wt,
                                                        float* __restrict__ Wt2,
@@ -523,11 +524,11 @@ __global__ void __launch_bounds__(256) k_lazy_update_w(int n_new, int m, int d, 
                                                        const float* __restrict__ U,
                                                        const float* __restrict__ C) {
     __shared__ float4 sC[BMAX][64];       // C[s][col0 .. col0+255]
-    __shared__ float sUr[BMAX][64];       // U[s][src[row]]
+    __shared__ __align__(16) float sUr[BMAX][64];       // U[s][src[row]]
     __shared__ int srow[64];
     const int l = blockIdx.z;
     const int i0 = blockIdx.x * 64, c0 = blockIdx.y * 256;
-    const int tid = threadIdx.x, tx = tid & 63, ty = tid >> 6;      // ty: rows ty, ty+4, ...
+    const int tid = threadIdx.x, tx = tid & 63, ty = tid >> 6;      // ty: rows 16 ty .. 16 ty + 15
     if (tid < 64) srow[tid] = (i0 + tid < n_new) ? src[(size_t)l * d + i0 + tid] : -1;
     __syncthreads();
     const float* Ul = U + (size_t)l * BMAX * d;
@@ -544,10 +545,10 @@ __global__ void __launch_bounds__(256) k_lazy_update_w(int n_new, int m, int d, 
     asm volatile("cp.async.commit_group;" ::: "memory");
     const int col = c0 + 4 * tx;
     const bool col_ok = col < rp;
-    float4 w[16];
+    float4 w[16];                                  // rows 16 ty + x of this CTA's 64
 #pragma unroll
     for (int x = 0; x < 16; ++x) {
-        const int sr = srow[ty + 4 * x];
+        const int sr = srow[16 * ty + x];
         w[x] = (sr >= 0 && col_ok)
                    ? __ldcs(reinterpret_cast<const float4*>(Wt + (size_t)l * d * rp + (size_t)sr * rp + col))
                    : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -557,16 +558,21 @@ __global__ void __launch_bounds__(256) k_lazy_update_w(int n_new, int m, int d, 
     for (int s = 0; s < m; ++s) {
         const float4 c = sC[s][tx];
 #pragma unroll
-        for (int x = 0; x < 16; ++x) {
-            const float nu = -sUr[s][ty + 4 * x];
-            w[x].x = fmaf(nu, c.x, w[x].x); w[x].y = fmaf(nu, c.y, w[x].y);
-            w[x].z = fmaf(nu, c.z, w[x].z); w[x].w = fmaf(nu, c.w, w[x].w);
+        for (int k = 0; k < 4; ++k) {
+            const float4 u4 = *reinterpret_cast<const float4*>(&sUr[s][16 * ty + 4 * k]);   // broadcast
+            const float nu[4] = {-u4.x, -u4.y, -u4.z, -u4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float4& t = w[4 * k + e];
+                t.x = fmaf(nu[e], c.x, t.x); t.y = fmaf(nu[e], c.y, t.y);
+                t.z = fmaf(nu[e], c.z, t.z); t.w = fmaf(nu[e], c.w, t.w);
+            }
         }
     }
     if (col_ok) {
 #pragma unroll
         for (int x = 0; x < 16; ++x) {
-            const int i = i0 + ty + 4 * x;
+            const int i = i0 + 16 * ty + x;
             if (i < n_new)
                 *reinterpret_cast<float4*>(Wt2 + (size_t)l * d * rp + (size_t)i * rp + col) = w[x];
         }

@@ -73,7 +73,7 @@ def test_hessian_zero_tokens_and_bad_args():
 
 
 # ------------------------------------------------------------------ damped inverse (a2, a3)
-@pytest.mark.parametrize("d,L", [(64, 1), (100, 2), (256, 3), (448, 1)])
+@pytest.mark.parametrize("d,L", [(64, 1), (100, 2), (256, 3), (448, 1), (827, 1), (1100, 2)])
 def test_damped_inverse_matches_oracle(d, L):
     z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=d, d_latent=max(8, d // 4),
