@@ -517,7 +517,7 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
 // A CTA owns 64 rows x 256 columns; the C panel and the rows' U entries are staged in shared
 // memory once per CTA, each thread carries 16 consecutive rows of one float4 column (per pending
 // step: one 128-bit load of C and four broadcast 128-bit loads of U for 64 FMAs).
-__global__ void __launch_bounds__(256) k_lazy_update_w(int n_new, int m, int d, int rp,
+__global__ void __launch_bounds__(256, 3) k_lazy_update_w(int n_new, int m, int d, int rp,
                                                        const float* __restrict__ Wt,
                                                        float* __restrict__ Wt2,
                                                        const int* __restrict__ src,
