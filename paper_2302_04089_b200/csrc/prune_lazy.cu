@@ -424,11 +424,15 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
     __shared__ __align__(16) float sZc[BMAX][64];
     __shared__ int srow[64], scol[64];
     const int l = blockIdx.y;
-    int ti = 0, rem = blockIdx.x;
-    while (rem > ti) { rem -= ti + 1; ++ti; }
-    const int tj = rem;
+    // linear index -> (ti, tj) of the lower triangle: ti = floor((sqrt(8 x + 1) - 1) / 2), fixed up
+    int ti = (int)((sqrtf(8.f * (float)blockIdx.x + 1.f) - 1.f) * 0.5f);
+    while (ti * (ti + 1) / 2 > (int)blockIdx.x) --ti;
+    while ((ti + 1) * (ti + 2) / 2 <= (int)blockIdx.x) ++ti;
+    const int tj = (int)blockIdx.x - ti * (ti + 1) / 2;
     const int i0 = ti * 64, j0 = tj * 64;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;     // rows 4ty + 32h + e, cols 4tx + e
+    // a tile strictly below the diagonal and inside the live range needs no per-entry checks
+    const bool interior = tj < ti && i0 + 64 <= n_new;
     const int* sl = src + (size_t)l * d;
     if (tid < 64) srow[tid] = (i0 + tid < n_new) ? sl[i0 + tid] : -1;
     else scol[tid - 64] = (j0 + tid - 64 < n_new) ? sl[j0 + tid - 64] : -1;
@@ -457,19 +461,31 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
 #pragma unroll
     for (int y = 0; y < 4; ++y) cs[y] = scol[4 * tx + y];
     float a[8][4], q[8][4];
+    if (interior) {
 #pragma unroll
-    for (int x = 0; x < 8; ++x) {
-        const int il = 4 * ty + 32 * (x >> 2) + (x & 3), i = i0 + il;
-        const int sr = srow[il];
-        const size_t roff = (size_t)(sr >= 0 ? sr : 0) * d;
+        for (int x = 0; x < 8; ++x) {
+            const unsigned roff = (unsigned)(srow[4 * ty + 32 * (x >> 2) + (x & 3)] * d);   // d * d < 2^31
 #pragma unroll
-        for (int y = 0; y < 4; ++y) {
-            const int j = j0 + 4 * tx + y;
-            if (sr >= 0 && j < i) {
-                a[x][y] = __ldcs(Al + roff + cs[y]);
-                q[x][y] = __ldcs(Ql + roff + cs[y]);
-            } else {
-                a[x][y] = 0.f; q[x][y] = 0.f;
+            for (int y = 0; y < 4; ++y) {
+                a[x][y] = __ldcs(Al + (roff + (unsigned)cs[y]));
+                q[x][y] = __ldcs(Ql + (roff + (unsigned)cs[y]));
+            }
+        }
+    } else {
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+            const int il = 4 * ty + 32 * (x >> 2) + (x & 3), i = i0 + il;
+            const int sr = srow[il];
+            const size_t roff = (size_t)(sr >= 0 ? sr : 0) * d;
+#pragma unroll
+            for (int y = 0; y < 4; ++y) {
+                const int j = j0 + 4 * tx + y;
+                if (sr >= 0 && j < i) {
+                    a[x][y] = __ldcs(Al + roff + cs[y]);
+                    q[x][y] = __ldcs(Ql + roff + cs[y]);
+                } else {
+                    a[x][y] = 0.f; q[x][y] = 0.f;
+                }
             }
         }
     }
@@ -499,6 +515,17 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
     float* Ao = A2 + (size_t)l * d * d;
     float* Qo = Q2 + (size_t)l * d * d;
     const int j = j0 + 4 * tx;
+    if (interior) {
+        float* ao = Ao + (size_t)(i0 + 4 * ty) * d + j;
+        float* qo = Qo + (size_t)(i0 + 4 * ty) * d + j;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+            const unsigned o = (unsigned)((32 * (x >> 2) + (x & 3)) * d);
+            *reinterpret_cast<float4*>(ao + o) = make_float4(a[x][0], a[x][1], a[x][2], a[x][3]);
+            *reinterpret_cast<float4*>(qo + o) = make_float4(q[x][0], q[x][1], q[x][2], q[x][3]);
+        }
+        return;
+    }
 #pragma unroll
     for (int x = 0; x < 8; ++x) {
         const int i = i0 + 4 * ty + 32 * (x >> 2) + (x & 3);
