@@ -25,16 +25,21 @@ static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratch
 namespace ziplm {
 namespace {
 constexpr int KC = 16;          // k-chunk staged in shared memory per pipeline stage
-constexpr int MT = 128;         // edge of the macro tile one CTA computes (2 x 2 tiles)
-constexpr int GT = 512;         // threads of a product CTA: 16 warps, 32 x 32 outputs per warp
+constexpr int MTM = 128;        // rows of the macro tile one CTA computes (two tiles)
+constexpr int MTN = 64;         // columns of the macro tile (one tile)
+constexpr int GT = 256;         // threads of a product CTA: 8 warps, 32 x 32 outputs per warp; two CTAs per SM
+constexpr int kSmallThreads = 512;   // threads of the base-case kernel
 constexpr int kStages = 3;      // cp.async pipeline depth
-// Shared-memory pitches (doubles).  Both are 4 mod 16, so that the 16 threads of a half-warp
-// (4 m-indices x 4 k-indices of an operand fragment) hit 16 different 8-byte banks, and both keep
+// Shared-memory pitches (doubles).  All are 4 mod 16, so that the 16 threads of a half-warp
+// (4 m-indices x 4 k-indices of an operand fragment) hit 16 different 8-byte banks, and all keep
 // rows 16-byte aligned for cp.async.
 constexpr int P_MK = KC + 4;    // chunk stored [m][k] (k contiguous in global memory)
-constexpr int P_KM = MT + 4;    // chunk stored [k][m] (m contiguous in global memory)
-constexpr int kStageDoubles = MT * P_MK > KC * P_KM ? MT * P_MK : KC * P_KM;
-constexpr size_t kProductSmemBytes = sizeof(double) * 2 * kStages * kStageDoubles;
+__host__ __device__ constexpr int pitch_km(int rows) { return rows + 4; }   // chunk stored [k][m] (m contiguous)
+__host__ __device__ constexpr int stage_doubles(int rows) {
+    return rows * P_MK > KC * pitch_km(rows) ? rows * P_MK : KC * pitch_km(rows);
+}
+constexpr int kStageA = stage_doubles(MTM), kStageB = stage_doubles(MTN);
+constexpr size_t kProductSmemBytes = sizeof(double) * kStages * (kStageA + kStageB);
 
 __device__ __forceinline__ void cp_async16(double* smem_dst, const double* gmem_src) {
     const unsigned sa = (unsigned)__cvta_generic_to_shared(smem_dst);
@@ -51,18 +56,19 @@ __device__ __forceinline__ void dmma884(double (&d)[2], double a, double b) {
                  : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
 }
 
-// Start the copy of one 128 x KC operand chunk into a pipeline stage; rows m >= m_valid (tiles
+// Start the copy of one ROWS x KC operand chunk into a pipeline stage; rows m >= m_valid (tiles
 // beyond the edge of the task) are not touched.
 //   KM == false: op(m,k) = P[m*ld + k], kept as s[m][k] (pitch P_MK);
-//   KM == true : op(m,k) = P[k*ld + m], kept as s[k][m] (pitch P_KM).
-template <bool KM>
+//   KM == true : op(m,k) = P[k*ld + m], kept as s[k][m] (pitch ROWS + 4).
+template <bool KM, int ROWS>
 __device__ __forceinline__ void chunk_async(double* s, const double* P, int ld, int k0, int m_valid) {
+    constexpr int PIECES = ROWS * KC / 2;                 // pieces of 16 bytes
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {
-        const int piece = threadIdx.x + e * GT;           // 1024 pieces of 16 bytes
+    for (int e = 0; e < PIECES / GT; ++e) {
+        const int piece = threadIdx.x + e * GT;
         if (KM) {
-            const int k = piece >> 6, m = (piece & 63) * 2;
-            if (m < m_valid) cp_async16(s + k * P_KM + m, P + (size_t)(k0 + k) * ld + m);
+            const int k = piece / (ROWS / 2), m = (piece % (ROWS / 2)) * 2;
+            if (m < m_valid) cp_async16(s + k * pitch_km(ROWS) + m, P + (size_t)(k0 + k) * ld + m);
         } else {
             const int m = piece >> 3, k = (piece & 7) * 2;
             if (m < m_valid) cp_async16(s + m * P_MK + k, P + (size_t)m * ld + k0 + k);
@@ -71,9 +77,9 @@ __device__ __forceinline__ void chunk_async(double* s, const double* P, int ld, 
 }
 
 // Operand fragment of the k-step kk (4 k's) for the 8 m-indices starting at m0.
-template <bool KM>
+template <bool KM, int ROWS>
 __device__ __forceinline__ double frag(const double* s, int m0, int kk, int lane) {
-    return KM ? s[(kk * 4 + (lane & 3)) * P_KM + m0 + (lane >> 2)]
+    return KM ? s[(kk * 4 + (lane & 3)) * pitch_km(ROWS) + m0 + (lane >> 2)]
               : s[(m0 + (lane >> 2)) * P_MK + kk * 4 + (lane & 3)];
 }
 
@@ -88,13 +94,13 @@ struct WarpAcc {
     }
 };
 
-// acc(128x128 macro tile) += opA(128xK) opB(Kx128) over the tile range [kt_lo, kt_hi) of K (in
+// acc(128 x 64 macro tile) += opA(128 x K) opB(K x 64) over the tile range [kt_lo, kt_hi) of K (in
 // tiles of 64), operands streamed through a three-stage cp.async pipeline with one barrier per
-// chunk.  Warp w owns rows 32 (w / 4) .. and columns 32 (w % 4) .. of the macro tile and only
+// chunk.  Warp w owns rows 32 (w / 2) .. and columns 32 (w % 2) .. of the macro tile and only
 // multiplies the chunks of its own range [my_lo, my_hi) (the triangular operands cut the range
 // per 64 x 64 tile; what the other warps' ranges bring into shared memory may be uninitialised
-// and is never read by this warp).  rows_valid / cols_valid crop the macro tile at the edge of
-// the task.  A and B point at k = 0 of the macro tile's rows / columns.
+// and is never read by this warp).  rows_valid crops the macro tile at the edge of the task.
+// A and B point at k = 0 of the macro tile's rows / columns.
 //   TA == false: A stored m x K row-major; true: stored K x m.
 //   TB == false: B stored K x n row-major; true: stored n x K.
 // The operand pointers are deliberately not __restrict__: callers read tiles written earlier in
@@ -102,18 +108,18 @@ struct WarpAcc {
 template <bool TA, bool TB>
 __device__ __forceinline__ void dgemm_macro(WarpAcc& acc, const double* A, int lda, const double* B,
                                             int ldb, int kt_lo, int kt_hi, int my_lo, int my_hi,
-                                            int rows_valid, int cols_valid, double* smem) {
+                                            int rows_valid, double* smem) {
     constexpr bool KA = TA, KB = !TB;       // orientation in memory: true = stored K x m
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int r0 = 32 * (warp >> 2), c0 = 32 * (warp & 3);
+    const int r0 = 32 * (warp >> 1), c0 = 32 * (warp & 1);
     double* sa = smem;
-    double* sb = smem + kStages * kStageDoubles;
+    double* sb = smem + kStages * kStageA;
     const int nchunks = (kt_hi - kt_lo) * (kTile / KC);
     const int kbase = kt_lo * kTile;
     for (int c = 0; c < kStages - 1; ++c) {
         if (c < nchunks) {
-            chunk_async<KA>(sa + c * kStageDoubles, A, lda, kbase + c * KC, rows_valid);
-            chunk_async<KB>(sb + c * kStageDoubles, B, ldb, kbase + c * KC, cols_valid);
+            chunk_async<KA, MTM>(sa + c * kStageA, A, lda, kbase + c * KC, rows_valid);
+            chunk_async<KB, MTN>(sb + c * kStageB, B, ldb, kbase + c * KC, MTN);
         }
         cp_async_commit();
     }
@@ -123,21 +129,21 @@ __device__ __forceinline__ void dgemm_macro(WarpAcc& acc, const double* A, int l
         const int nx = c + kStages - 1;
         if (nx < nchunks) {
             const int st = nx % kStages;
-            chunk_async<KA>(sa + st * kStageDoubles, A, lda, kbase + nx * KC, rows_valid);
-            chunk_async<KB>(sb + st * kStageDoubles, B, ldb, kbase + nx * KC, cols_valid);
+            chunk_async<KA, MTM>(sa + st * kStageA, A, lda, kbase + nx * KC, rows_valid);
+            chunk_async<KB, MTN>(sb + st * kStageB, B, ldb, kbase + nx * KC, MTN);
         }
         cp_async_commit();
         const int ktile = kt_lo + c / (kTile / KC);
         if (ktile < my_lo || ktile >= my_hi) continue;
-        const double* pa = sa + (c % kStages) * kStageDoubles;
-        const double* pb = sb + (c % kStages) * kStageDoubles;
+        const double* pa = sa + (c % kStages) * kStageA;
+        const double* pb = sb + (c % kStages) * kStageB;
 #pragma unroll
         for (int kk = 0; kk < KC / 4; ++kk) {
             double a[4], b[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                a[i] = frag<KA>(pa, r0 + 8 * i, kk, lane);
-                b[i] = frag<KB>(pb, c0 + 8 * i, kk, lane);
+                a[i] = frag<KA, MTM>(pa, r0 + 8 * i, kk, lane);
+                b[i] = frag<KB, MTN>(pb, c0 + 8 * i, kk, lane);
             }
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -148,12 +154,23 @@ __device__ __forceinline__ void dgemm_macro(WarpAcc& acc, const double* A, int l
     cp_async_wait<0>();
 }
 
-// Linear index -> (row, col) of the lower triangle, rows in order 0, 1, ...
-__device__ __forceinline__ void lower_index(int idx, int& row, int& col) {
-    row = 0;
-    while (idx > row) { idx -= row + 1; ++row; }
-    col = idx;
+// Macro tiles (I, J) of a lower-triangular region of T x T tiles: row block I (tiles 2I, 2I+1)
+// meets the column tiles J <= 2I + 1.  Count, and linear index -> (I, J) in row-block order.
+__host__ __device__ inline int lower_macro_count(int T) {
+    int n = 0;
+    for (int I = 0; 2 * I < T; ++I) n += (2 * I + 2 < T) ? 2 * I + 2 : T;
+    return n;
 }
+__device__ __forceinline__ void lower_macro_index(int idx, int T, int& I, int& J) {
+    I = 0;
+    for (;;) {
+        const int w = (2 * I + 2 < T) ? 2 * I + 2 : T;
+        if (idx < w) break;
+        idx -= w; ++I;
+    }
+    J = idx;
+}
+
 
 // lambda[l] = damp_frac * mean(diag H[l]); flags non-finite diagonals and non-positive means.
 __global__ void __launch_bounds__(256) k_mean_diag(const float* __restrict__ H, int d,
@@ -243,47 +260,46 @@ __device__ __forceinline__ void task_krange(const GemmTask& t, int ti, int tj, i
     else if (t.kmode == 3) klo = tj;
 }
 
-// One CTA per 128 x 128 macro tile (2 x 2 tiles); blockIdx.x runs over the macro tiles of the
-// task (the lower triangle of macro tiles when lower_only), blockIdx.y over the layers.
+// One CTA per 128 x 64 macro tile (two tiles high); blockIdx.x runs over the macro tiles of the
+// task (those that reach the lower triangle when lower_only), blockIdx.y over the layers.
 template <bool TA, bool TB>
-__global__ void __launch_bounds__(GT, 1) k_dgemm_tiles(GemmTask t, int dp) {
+__global__ void __launch_bounds__(GT, 2) k_dgemm_tiles(GemmTask t, int dp) {
     extern __shared__ __align__(16) double smem[];
     const int l = blockIdx.y;
-    const int mmt = (t.mt + 1) / 2, nmt = (t.nt + 1) / 2;
+    const int mmt = (t.mt + 1) / 2;
     // macro tiles with the longest k range come first, so that the last wave is the lightest
     int I, J;
-    if (t.lower_only) lower_index(blockIdx.x, I, J);
-    else if (t.kmode == 1) { J = nmt - 1 - blockIdx.x / mmt; I = blockIdx.x % mmt; }
+    if (t.lower_only) lower_macro_index(blockIdx.x, t.mt, I, J);
+    else if (t.kmode == 1) { J = t.nt - 1 - blockIdx.x / mmt; I = blockIdx.x % mmt; }
     else if (t.kmode == 3) { J = blockIdx.x / mmt; I = blockIdx.x % mmt; }
-    else if (t.kmode == 2) { I = mmt - 1 - blockIdx.x / nmt; J = blockIdx.x % nmt; }
-    else { I = blockIdx.x / nmt; J = blockIdx.x % nmt; }
+    else if (t.kmode == 2) { I = mmt - 1 - blockIdx.x / t.nt; J = blockIdx.x % t.nt; }
+    else { I = blockIdx.x / t.nt; J = blockIdx.x % t.nt; }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ti = 2 * I + (warp >> 3), tj = 2 * J + ((warp >> 1) & 1);   // this warp's tile
-    const bool mine = ti < t.mt && tj < t.nt && (!t.lower_only || ti >= tj);
+    const int ti = 2 * I + (warp >> 2), tj = J;                          // this warp's tile
+    const bool mine = ti < t.mt && (!t.lower_only || ti >= tj);
     // CTA range: union over its valid tiles; warp range: its own tile's
     int kt_lo = t.kt, kt_hi = 0;
-    for (int a = 0; a < 2; ++a)
-        for (int b = 0; b < 2; ++b) {
-            const int si = 2 * I + a, sj = 2 * J + b;
-            if (si >= t.mt || sj >= t.nt || (t.lower_only && si < sj)) continue;
-            int lo, hi;
-            task_krange(t, si, sj, lo, hi);
-            kt_lo = min(kt_lo, lo); kt_hi = max(kt_hi, hi);
-        }
+    for (int a = 0; a < 2; ++a) {
+        const int si = 2 * I + a;
+        if (si >= t.mt || (t.lower_only && si < tj)) continue;
+        int lo, hi;
+        task_krange(t, si, tj, lo, hi);
+        kt_lo = min(kt_lo, lo); kt_hi = max(kt_hi, hi);
+    }
     int my_lo = 0, my_hi = 0;
     if (mine) task_krange(t, ti, tj, my_lo, my_hi);
-    const int rows_valid = min(MT, (t.mt - 2 * I) * kTile), cols_valid = min(MT, (t.nt - 2 * J) * kTile);
+    const int rows_valid = min(MTM, (t.mt - 2 * I) * kTile);
     const size_t lay = (size_t)l * dp * dp;
     const double* A = t.A + lay + (TA ? ((size_t)t.a_r * kTile * dp + (size_t)(t.a_c + 2 * I) * kTile)
                                       : ((size_t)(t.a_r + 2 * I) * kTile * dp + (size_t)t.a_c * kTile));
-    const double* B = t.B + lay + (TB ? ((size_t)(t.b_r + 2 * J) * kTile * dp + (size_t)t.b_c * kTile)
-                                      : ((size_t)t.b_r * kTile * dp + (size_t)(t.b_c + 2 * J) * kTile));
+    const double* B = t.B + lay + (TB ? ((size_t)(t.b_r + J) * kTile * dp + (size_t)t.b_c * kTile)
+                                      : ((size_t)t.b_r * kTile * dp + (size_t)(t.b_c + J) * kTile));
     WarpAcc acc;
     acc.zero();
-    dgemm_macro<TA, TB>(acc, A, dp, B, dp, kt_lo, kt_hi, my_lo, my_hi, rows_valid, cols_valid, smem);
+    dgemm_macro<TA, TB>(acc, A, dp, B, dp, kt_lo, kt_hi, my_lo, my_hi, rows_valid, smem);
     if (!mine) return;
-    double* out = t.C + lay + (size_t)((t.c_r + 2 * I) * kTile + 32 * (warp >> 2)) * dp +
-                  (size_t)(t.c_c + 2 * J) * kTile + 32 * (warp & 3);
+    double* out = t.C + lay + (size_t)((t.c_r + 2 * I) * kTile + 32 * (warp >> 1)) * dp +
+                  (size_t)(t.c_c + J) * kTile + 32 * (warp & 1);
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -313,7 +329,7 @@ struct SmallSmem {
 __device__ __forceinline__ void tile_async(double* dst, const double* src, int ld) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const int piece = threadIdx.x + e * GT;            // 2048 pieces of 16 bytes
+        const int piece = threadIdx.x + e * kSmallThreads;            // 2048 pieces of 16 bytes
         const int r = piece >> 5, c = (piece & 31) * 2;
         cp_async16(dst + r * PS + c, src + (size_t)r * ld + c);
     }
@@ -418,7 +434,7 @@ __device__ __forceinline__ void leaf_factor(const double* Ag, double* Fg, double
     __syncthreads();                          // earlier readers of the shared arrays are done
     tile_async(sm.tb, Ag, dp);
     cp_async_commit();
-    for (int e = tid; e < kTile * PS; e += GT) sm.ta[e] = 0.0;   // the inverse is built in ta
+    for (int e = tid; e < kTile * PS; e += kSmallThreads) sm.ta[e] = 0.0;   // the inverse is built in ta
     cp_async_wait<0>();
     __syncthreads();
     double r[4][4];
@@ -535,7 +551,7 @@ __device__ __forceinline__ void leaf_factor(const double* Ag, double* Fg, double
         warp_store16(acc, sm.ta + rb * PS + cb, PS, -1.0);
     }
     __syncthreads();
-    for (int e = tid; e < kTile * kTile; e += GT) {
+    for (int e = tid; e < kTile * kTile; e += kSmallThreads) {
         const int i = e >> 6, jj = e & 63;
         const double m = sm.ta[i * PS + jj];
         Fg[(size_t)i * dp + jj] = (jj <= i) ? sm.s[i][jj] : 0.0;
@@ -549,7 +565,7 @@ __device__ __forceinline__ void leaf_factor(const double* Ag, double* Fg, double
 // right-looking tile Cholesky (A -> F) followed by the block forward substitution for M = F^-1.
 // Every product is a 64 x 64 x 64 tile product of the whole CTA on the float64 tensor core, with
 // its operands fetched from global memory (the L2) into shared memory.
-__global__ void __launch_bounds__(GT, 1) k_factor_small(double* A, double* F, double* M, int dp, int lo,
+__global__ void __launch_bounds__(kSmallThreads, 1) k_factor_small(double* A, double* F, double* M, int dp, int lo,
                                                         int nt, int* layer_status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SmallSmem& sm = *reinterpret_cast<SmallSmem*>(smem_raw);
@@ -629,26 +645,26 @@ __global__ void __launch_bounds__(GT, 1) k_factor_small(double* A, double* F, do
 
 // H^-1 = M^T M on the lower tiles (i >= j): sum over k >= i of M_ki^T M_kj; writes the cropped
 // d x d result as float64 (mirrored to the upper triangle) and/or fp32 strict lower + fp64 diag.
-// One CTA per 128 x 128 macro tile of the lower triangle.
-__global__ void __launch_bounds__(GT, 1) k_lauum(const double* M, int dp, int T, int d, double* out64,
+// One CTA per 128 x 64 macro tile that reaches the lower triangle.
+__global__ void __launch_bounds__(GT, 2) k_lauum(const double* M, int dp, int T, int d, double* out64,
                                                  float* tri32, int pitch32, double* diag64) {
     extern __shared__ __align__(16) double smem[];
     const int l = blockIdx.y;
     int I, J;
-    lower_index(blockIdx.x, I, J);
+    lower_macro_index(blockIdx.x, T, I, J);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ti = 2 * I + (warp >> 3), tj = 2 * J + ((warp >> 1) & 1);
-    const bool mine = ti < T && tj < T && ti >= tj;
+    const int ti = 2 * I + (warp >> 2), tj = J;
+    const bool mine = ti < T && ti >= tj;
     const double* Ml = M + (size_t)l * dp * dp;
-    const int rows_valid = min(MT, (T - 2 * I) * kTile), cols_valid = min(MT, (T - 2 * J) * kTile);
+    const int rows_valid = min(MTM, (T - 2 * I) * kTile);
     WarpAcc acc;
     acc.zero();
     // (M^T M)_ij: opA(i,k) = M[k][i] (stored K x m), opB(k,j) = M[k][j]; tile (ti, .) starts at k = ti
-    dgemm_macro<true, false>(acc, Ml + (size_t)(2 * I) * kTile, dp, Ml + (size_t)(2 * J) * kTile, dp,
-                             2 * I, T, mine ? ti : 0, mine ? T : 0, rows_valid, cols_valid, smem);
+    dgemm_macro<true, false>(acc, Ml + (size_t)(2 * I) * kTile, dp, Ml + (size_t)J * kTile, dp,
+                             2 * I, T, mine ? ti : 0, mine ? T : 0, rows_valid, smem);
     if (!mine) return;
-    const int row0 = 2 * I * kTile + 32 * (warp >> 2) + (lane >> 2);
-    const int col0 = 2 * J * kTile + 32 * (warp & 3) + 2 * (lane & 3);
+    const int row0 = 2 * I * kTile + 32 * (warp >> 1) + (lane >> 2);
+    const int col0 = J * kTile + 32 * (warp & 1) + 2 * (lane & 3);
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -680,8 +696,8 @@ struct InvCtx {
 
 template <bool TA, bool TB>
 ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
-    const int mm = (t.mt + 1) / 2, nm = (t.nt + 1) / 2;      // macro tiles
-    const int ctas = t.lower_only ? mm * (mm + 1) / 2 : mm * nm;
+    const int mm = (t.mt + 1) / 2;                           // macro tiles: mm x t.nt
+    const int ctas = t.lower_only ? lower_macro_count(t.mt) : mm * t.nt;
     if (ctas <= 0 || t.kt <= 0) return ZIPLM_OK;
     static const cudaError_t attr = cudaFuncSetAttribute(
         k_dgemm_tiles<TA, TB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
@@ -700,7 +716,7 @@ ziplm_status factor_range(const InvCtx& c, int lo, int hi) {
             k_factor_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmallSmem));
         if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
         PhaseScope ps(PH_INV_LEAVES, c.st);
-        k_factor_small<<<c.L, GT, sizeof(SmallSmem), c.st>>>(c.A, c.F, c.M, c.dp, lo, hi - lo,
+        k_factor_small<<<c.L, kSmallThreads, sizeof(SmallSmem), c.st>>>(c.A, c.F, c.M, c.dp, lo, hi - lo,
                                                               c.layer_status);
         ZIPLM_CHECK_LAUNCH();
         return ZIPLM_OK;
@@ -761,9 +777,8 @@ ziplm_status run_damped_inverse(const float* H, int L, int d, float damp_frac, d
         static const cudaError_t attr = cudaFuncSetAttribute(
             k_lauum, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
         if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
-        const int Tm = (T + 1) / 2;
-        k_lauum<<<dim3(Tm * (Tm + 1) / 2, L), GT, kProductSmemBytes, st>>>(ctx.M, dp, T, d, out64, tri32,
-                                                                         pitch32, diag64);
+        k_lauum<<<dim3(lower_macro_count(T), L), GT, kProductSmemBytes, st>>>(ctx.M, dp, T, d, out64, tri32,
+                                                                            pitch32, diag64);
         ZIPLM_CHECK_LAUNCH();
     }
     if (lam_out) {
