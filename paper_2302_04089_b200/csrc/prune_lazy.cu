@@ -141,9 +141,13 @@ __device__ __forceinline__ Cand bcast_cand(const Cand& c, int src_lane) {
 // the lanes within 1e-5 of the fp32 minimum (almost always a single one) go through the exact
 // float64 comparison, so the common case costs six 32-bit shuffles instead of five rounds of
 // 64-bit exchanges.
-__device__ __forceinline__ Cand warp_best(const Cand& mine) {
-    float r = INFINITY;
-    if (mine.pos >= 0) r = cand_valid(mine) ? (float)mine.q / (float)mine.a : -INFINITY;
+// fp32 quotient that orders candidates coarsely: +inf for "none", -inf for an invalid entry.
+__device__ __forceinline__ float cand_quotient(const Cand& c) {
+    if (c.pos < 0) return INFINITY;
+    return cand_valid(c) ? __fdividef((float)c.q, (float)c.a) : -INFINITY;
+}
+
+__device__ __forceinline__ Cand warp_best(const Cand& mine, float r) {
     float rmin = r;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) rmin = fminf(rmin, __shfl_xor_sync(0xffffffffu, rmin, off));
@@ -158,6 +162,8 @@ __device__ __forceinline__ Cand warp_best(const Cand& mine) {
     }
     return best;
 }
+
+__device__ __forceinline__ Cand warp_best(const Cand& mine) { return warp_best(mine, cand_quotient(mine)); }
 
 // nsteps greedy steps of one layer, run by a thread-block cluster of CS CTAs (CS = 1, 2, 4 or 8,
 // chosen so that a CTA's slice of positions fits its shared memory).  CTA `rank` owns the
@@ -192,7 +198,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
     extern __shared__ float4 dyn_smem4[];
     float* sU = reinterpret_cast<float*>(dyn_smem4);       // [BMAX][S]
     float* sZ = sU + (size_t)BMAX * S;                     // [BMAX][S]
-    __shared__ Cand s_cand[2][NW];                         // per-warp candidates, by step parity
+    __shared__ Cand s_cand[2][CLUSTER_MAX * NW];           // all warps of the cluster, by step parity
     __shared__ float sT[BMAX][BMAX];                       // T[m][s] = u_s[p_m]
     __shared__ float sUp[BMAX], sZp[BMAX];
     __shared__ int s_pm[BMAX];
@@ -225,28 +231,39 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
 
     for (int m = 0; m < nsteps; ++m) {
         const int par = m & 1;
-        // ---- per-warp best of rho = Q[k,k] / H^-1[k,k] (ties: lowest original index)
+        // ---- per-warp best of rho = Q[k,k] / H^-1[k,k] (ties: lowest original index).  The four
+        //      owned positions are ordered by an fp32 quotient; only those within 1e-5 of the
+        //      smallest (almost always one) go through the exact float64 comparison.
         Cand best;
         best.a = 1.0; best.q = 0.0; best.org = 0x7fffffff; best.pos = -1;
+        float rq[4], rbest = INFINITY;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            if (!alive[e]) continue;
+            rq[e] = INFINITY;
+            if (alive[e]) {
+                const bool ok = da[e] > 0.0 && isfinite(da[e]) && isfinite(dq[e]);
+                rq[e] = ok ? __fdividef((float)dq[e], (float)da[e]) : -INFINITY;
+            }
+            rbest = fminf(rbest, rq[e]);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (!alive[e] || !(rq[e] == rbest || rq[e] <= rbest + fabsf(rbest) * 1e-5f)) continue;
             Cand c;
             c.a = da[e]; c.q = dq[e]; c.org = org[e]; c.pos = k0 + e;
             merge_cand(best, c);
         }
-        best = warp_best(best);
-        if (lane == 0) s_cand[par][warp] = best;
+        best = warp_best(best, best.pos >= 0 ? rbest : INFINITY);
+        // push: lane c < CS hands the warp's candidate to CTA c, so that after the barrier every
+        // CTA finds all candidates in its own shared memory
+        if (lane < CS) *cluster.map_shared_rank(&s_cand[par][rank * NW + warp], lane) = best;
         cluster.sync();
         // ---- warp 0 of every CTA: global pick from all warps of all CTAs, then the pending
         //      vectors' entries at the pivot (from the CTA that owns it)
         if (warp == 0) {
             Cand g;
             g.a = 1.0; g.q = 0.0; g.org = 0x7fffffff; g.pos = -1;
-            for (int e = lane; e < CS * NW; e += 32) {
-                const Cand* remote = cluster.map_shared_rank(&s_cand[par][e % NW], e / NW);
-                merge_cand(g, *remote);
-            }
+            for (int e = lane; e < CS * NW; e += 32) merge_cand(g, s_cand[par][e]);
             g = warp_best(g);
             int p = g.pos;
             if (p < 0) p = 0;
@@ -284,8 +301,6 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
         const double rs = s_rs, half = s_half;
         // ---- true pivot columns of H^-1 and Q on the owned positions; float64 diagonal downdate
         if (owner_thread) {
-            // The pending terms are subtracted with fp32 FMAs, one rounding per term: exactly
-            // what the per-step streaming variant does to the stored entry.
             float a[4], q[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -297,6 +312,8 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
                     q[e] = Ql[off];
                 }
             }
+            // pending terms at the pivot, summed while the gathered entries are still in flight
+            float ca[4] = {0.f, 0.f, 0.f, 0.f}, cq[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 4
             for (int s = 0; s < m; ++s) {
                 const float4 u4 = *reinterpret_cast<const float4*>(sU + (size_t)s * S + kloc);
@@ -305,11 +322,13 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
                 const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, zz[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    a[e] = fmaf(-uu[e], up, a[e]);
-                    q[e] = fmaf(-zz[e], up, q[e]);
-                    q[e] = fmaf(-uu[e], zp, q[e]);
+                    ca[e] = fmaf(uu[e], up, ca[e]);
+                    cq[e] = fmaf(zz[e], up, cq[e]);
+                    cq[e] = fmaf(uu[e], zp, cq[e]);
                 }
             }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { a[e] -= ca[e]; q[e] -= cq[e]; }
             float u32[4], z32[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
