@@ -644,7 +644,8 @@ __global__ void __launch_bounds__(kSmallThreads, 1) k_factor_small(double* A, do
 }
 
 // H^-1 = M^T M on the lower tiles (i >= j): sum over k >= i of M_ki^T M_kj; writes the cropped
-// d x d result as float64 (mirrored to the upper triangle) and/or fp32 strict lower + fp64 diag.
+// d x d result as float64 (mirrored to the upper triangle) and/or fp32 off-diagonal (both
+// triangles) + fp64 diag.
 // One CTA per 128 x 64 macro tile that reaches the lower triangle.
 __global__ void __launch_bounds__(GT, 2) k_lauum(const double* M, int dp, int T, int d, double* out64,
                                                  float* tri32, int pitch32, double* diag64) {
@@ -679,8 +680,11 @@ __global__ void __launch_bounds__(GT, 2) k_lauum(const double* M, int dp, int T,
                     o[(size_t)row * d + col] = v;
                     o[(size_t)col * d + row] = v;
                 }
-                if (tri32 && row > col)
-                    tri32[(size_t)l * d * pitch32 + (size_t)row * pitch32 + col] = (float)v;
+                if (tri32 && row > col) {       // both triangles: a column can then be read as a row
+                    float* t = tri32 + (size_t)l * d * pitch32;
+                    t[(size_t)row * pitch32 + col] = (float)v;
+                    t[(size_t)col * pitch32 + row] = (float)v;
+                }
                 if (diag64 && row == col) diag64[(size_t)l * d + row] = v;
             }
 }

@@ -23,7 +23,7 @@
 // independent, so no grid-wide synchronisation is needed) and two update kernels.  Block boundaries are placed on
 // the requested levels, where W is up to date and can be snapshotted.
 //
-// Layout per layer: A, Q fp32 [d, d] strict lower triangles (two buffers each, ping-pong),
+// Layout per layer: A, Q fp32 [d, d], off-diagonal entries in both triangles (two buffers each, ping-pong),
 // Wt = W^T fp32 [d, rp] (two buffers), float64 diagonals, pending U, Z [B, d] and C [B, rp].
 #include <cooperative_groups.h>
 #include <math.h>
@@ -301,17 +301,13 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
         const double rs = s_rs, half = s_half;
         // ---- true pivot columns of H^-1 and Q on the owned positions; float64 diagonal downdate
         if (owner_thread) {
-            float a[4], q[4];
+            // both triangles of H^-1 and Q are kept, so the pivot column is the contiguous row p
+            const float4 a4 = *reinterpret_cast<const float4*>(Al + (size_t)p * d + k0);
+            const float4 q4 = *reinterpret_cast<const float4*>(Ql + (size_t)p * d + k0);
+            float a[4] = {a4.x, a4.y, a4.z, a4.w}, q[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int k = k0 + e;
-                a[e] = 0.f; q[e] = 0.f;
-                if (alive[e] && k != p) {
-                    const size_t off = (k < p) ? ((size_t)p * d + k) : ((size_t)k * d + p);
-                    a[e] = Al[off];
-                    q[e] = Ql[off];
-                }
-            }
+            for (int e = 0; e < 4; ++e)
+                if (!alive[e] || k0 + e == p) { a[e] = 0.f; q[e] = 0.f; }
             // pending terms at the pivot, summed while the gathered entries are still in flight
             float ca[4] = {0.f, 0.f, 0.f, 0.f}, cq[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 4
@@ -424,23 +420,24 @@ __device__ __forceinline__ void cp_async16_zfill(float4* smem_dst, const float* 
                  : "memory");
 }
 
-// Rank-m update of the strict lower triangles of H^-1 and Q with compaction (out of place):
+// Rank-m update of the off-diagonal entries of H^-1 and Q with compaction (out of place):
 //   A'[i,j] = A[si,sj] - sum_s U[s,si] U[s,sj],
 //   Q'[i,j] = Q[si,sj] - sum_s (Z[s,si] U[s,sj] + U[s,si] Z[s,sj]),    si = src[i] > sj = src[j].
 // 64 x 64 tiles of the new index space, 128 threads, 8 rows x 4 columns of both matrices per
-// thread: per pending step six 128-bit shared-memory loads feed 96 FMAs.  Entries above the
-// diagonal of a tile that straddles it are written too (the upper triangles are never read).
-__global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
+// thread: per pending step six 128-bit shared-memory loads feed 96 FMAs.  Every entry is stored
+// twice, at [i][j] and [j][i]: the steps kernel reads a pivot column as a contiguous row.
+__global__ void __launch_bounds__(128, 5) k_lazy_update_aq(int n_new, int m, int d,
                                                         const float* __restrict__ A,
                                                         const float* __restrict__ Q,
                                                         float* __restrict__ A2, float* __restrict__ Q2,
                                                         const int* __restrict__ src,
                                                         const float* __restrict__ U,
                                                         const float* __restrict__ Z) {
-    __shared__ __align__(16) float sUr[BMAX][64];
-    __shared__ __align__(16) float sZr[BMAX][64];
-    __shared__ __align__(16) float sUc[BMAX][64];
-    __shared__ __align__(16) float sZc[BMAX][64];
+    __shared__ __align__(16) float stage[4][BMAX][64];   // pending slabs of the tile's rows and columns
+    float (*sUr)[64] = stage[0];
+    float (*sZr)[64] = stage[1];
+    float (*sUc)[64] = stage[2];
+    float (*sZc)[64] = stage[3];
     __shared__ int srow[64], scol[64];
     const int l = blockIdx.y;
     // linear index -> (ti, tj) of the lower triangle: ti = floor((sqrt(8 x + 1) - 1) / 2), fixed up
@@ -543,19 +540,36 @@ __global__ void __launch_bounds__(128) k_lazy_update_aq(int n_new, int m, int d,
             *reinterpret_cast<float4*>(ao + o) = make_float4(a[x][0], a[x][1], a[x][2], a[x][3]);
             *reinterpret_cast<float4*>(qo + o) = make_float4(q[x][0], q[x][1], q[x][2], q[x][3]);
         }
+        // mirror ([j][i]): the tile goes through shared memory (the staging arrays are free now),
+        // so that the transposed rows leave as contiguous 256-byte pieces
+        float* tbuf = &stage[0][0][0];                 // 64 x 65 floats of the 4 x 32 x 64
+        const int lane = tid & 31, wrp = tid >> 5;
+#pragma unroll
+        for (int mat = 0; mat < 2; ++mat) {
+            __syncthreads();                           // the arrays' previous readers are done
+#pragma unroll
+            for (int x = 0; x < 8; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y)
+                    tbuf[(4 * tx + y) * 65 + 4 * ty + 32 * (x >> 2) + (x & 3)] = mat ? q[x][y] : a[x][y];
+            __syncthreads();
+            float* mo = (mat ? Qo : Ao) + (size_t)j0 * d + i0 + 2 * lane;
+#pragma unroll 4
+            for (int jl = wrp; jl < 64; jl += 4)
+                *reinterpret_cast<float2*>(mo + (size_t)jl * d) =
+                    make_float2(tbuf[jl * 65 + 2 * lane], tbuf[jl * 65 + 2 * lane + 1]);
+        }
         return;
     }
 #pragma unroll
     for (int x = 0; x < 8; ++x) {
         const int i = i0 + 4 * ty + 32 * (x >> 2) + (x & 3);
         if (i >= n_new || j >= i) continue;
-        if (j + 3 >= d) {
-            for (int e = 0; e < 4; ++e)
-                if (j + e < i) { Ao[(size_t)i * d + j + e] = a[x][e]; Qo[(size_t)i * d + j + e] = q[x][e]; }
-        } else {
-            *reinterpret_cast<float4*>(Ao + (size_t)i * d + j) = make_float4(a[x][0], a[x][1], a[x][2], a[x][3]);
-            *reinterpret_cast<float4*>(Qo + (size_t)i * d + j) = make_float4(q[x][0], q[x][1], q[x][2], q[x][3]);
-        }
+        for (int e = 0; e < 4; ++e)          // tile on the diagonal or at the ragged edge: entry by entry
+            if (j + e < i) {
+                Ao[(size_t)i * d + j + e] = a[x][e]; Ao[(size_t)(j + e) * d + i] = a[x][e];
+                Qo[(size_t)i * d + j + e] = q[x][e]; Qo[(size_t)(j + e) * d + i] = q[x][e];
+            }
     }
 }
 

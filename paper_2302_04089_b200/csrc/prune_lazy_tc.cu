@@ -12,7 +12,8 @@
 // thread issues the 48 tcgen05.mma of the three split products (hi*hi and the cross terms in
 // accumulators of their own, all starting from zero), and eight epilogue warps read the
 // accumulators back, transpose them through shared memory so that lanes run along a matrix row,
-// and subtract them from the gathered old entries with one fp32 operation each.  The kernel is
+// and subtract them from the gathered old entries with one fp32 operation each; every entry is
+// stored at [i][j] and at [j][i].  The kernel is
 // left with the streaming of the two triangles; two CTAs per SM overlap each other's phases.
 //
 // Every mbarrier wait is bounded; a wait that runs out marks the layer ZIPLM_ERR_TIMEOUT and the
@@ -210,12 +211,22 @@ k_lazy_update_aq_tc(const __grid_constant__ CUtensorMap map, int n_new, int d,
                     tb[lane * 33 + h * 16 + e] = __uint_as_float(v[e]) + __uint_as_float(w[e]);
             }
             __syncwarp();
-            float* prow = (mat ? Q2 : A2) + (size_t)l * d * d + (size_t)ibase * d + j;
+            float* Mo = (mat ? Q2 : A2) + (size_t)l * d * d;
+            float* prow = Mo + (size_t)ibase * d + j;
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
                 const float val = (mat ? cq[e] : ca[e]) - tb[e * 33 + lane];
+                tb[e * 33 + lane] = val;
                 if (ibase + e < n_new && j < ibase + e) prow[0] = val;
                 prow += d;
+            }
+            __syncwarp();
+            // mirror ([j][i]): back in the row-per-lane view, so that lanes run along i
+            float* pcol = Mo + (size_t)(j0 + cc * 32) * d + ibase + lane;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+                if (ibase + lane < n_new && j0 + cc * 32 + e < ibase + lane) pcol[0] = tb[lane * 33 + e];
+                pcol += d;
             }
             __syncwarp();
         }
