@@ -175,10 +175,10 @@ LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in p
 # since the captures.
 NCU_TRAFFIC = {
     # k_lazy_update_aq, first block (n_new = 3040): profiles/k_lazy_kernels_c3_4layers.md
-    "k_lazy_update_aq": dict(bytes=3 * (164.0e6 + 90.1e6), launch="n_new = 3040, m = 32",
-                             algorithmic=12 * 16.0 * 3040 * 3039 / 2),
+    "k_lazy_update_aq": dict(bytes=3 * (169.8e6 + 235.8e6), launch="n_new = 3040, m = 32",
+                             algorithmic=12 * 24.0 * 3040 * 3039 / 2),
     # k_dgemm_tiles, top-level product F21 = A21 M11^T: profiles/inverse_kernels_c3.md
-    "k_dgemm_tiles": dict(bytes=3 * (116.7e6 + 47.3e6), launch="F21 = A21 M11^T, 12 x 12 macro tiles",
+    "k_dgemm_tiles": dict(bytes=3 * (116.3e6 + 49.6e6), launch="F21 = A21 M11^T, 12 x 24 macro tiles",
                           algorithmic=None),
     # k_neuron_update at n = 3066: profiles/k_neuron_update_c3_4layers.md
     "k_neuron_update": dict(bytes=3 * (113.8e6 + 56.6e6), launch="n = 3066",
@@ -188,8 +188,9 @@ NCU_TRAFFIC = {
 
 def lazy_update_work(L, G, levels):
     """Algorithmic work of k_lazy_update_aq over one greedy run: a launch that leaves n live
-    structures reads and writes the strict lower triangles of H^-1 and Q once (2 matrices x
-    n(n-1)/2 entries x 4 B x (read + write)) and spends 3 fp32 FMA per entry and pending step.
+    structures reads the off-diagonal entries of H^-1 and Q once per symmetric pair and writes
+    them at [i][j] and [j][i] (2 matrices x n(n-1)/2 pairs x 4 B x (1 read + 2 writes)) and spends
+    3 fp32 FMA per pair and pending step.
     Block boundaries fall on the requested levels, as in the library.  Returns (bytes, fma,
     launches)."""
     n, slot, nbytes, fma, launches = G, 0, 0.0, 0.0, 0
@@ -201,7 +202,7 @@ def lazy_update_work(L, G, levels):
         n -= m
         if n > 1:
             entries = L * n * (n - 1) / 2.0
-            nbytes += 16.0 * entries
+            nbytes += 24.0 * entries
             fma += 3.0 * m * entries
             launches += 1
         if slot < len(levels) and levels[slot] == n:
