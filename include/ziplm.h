@@ -11,7 +11,7 @@
  *     stream) and the call returns without synchronising: it starts after everything already
  *     enqueued there and the stream continues only when it is complete.  Buffers must stay alive
  *     until the stream has drained.  ziplm_prune_layers may run groups of layers concurrently on
- *     up to four internal non-blocking streams (created once per device, on first use), forked
+ *     up to eight internal non-blocking streams (created once per device, on first use), forked
  *     from and joined back to `cuda_stream` with events.
  *   - The return value reports what the host can see when the work is enqueued (bad arguments,
  *     workspace too small, a failed launch).  Failures that depend on the data (a Hessian that
