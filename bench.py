@@ -287,10 +287,31 @@ def run_ours(args, shape):
     h2d = Wh.numel() * 4 + Xh.numel() * Xh.element_size()
     d2h = sum(v.numel() * v.element_size() for v in host_out.values())
 
+    # The upload of X is the longest part of this leg, so it is pipelined with the Hessian through
+    # the same public calls: X goes up in chunks of layers on a copy stream and the Hessian of a
+    # chunk is enqueued as soon as its activations have arrived.
+    copy_stream = torch.cuda.Stream()
+    n_chunks = min(4, L)
+    bounds = [L * c // n_chunks for c in range(n_chunks + 1)]
+
     def e2e_step():
-        W.copy_(Wh, non_blocking=True)
-        X.copy_(Xh, non_blocking=True)
-        step()
+        nonlocal out
+        cur = torch.cuda.current_stream()
+        copy_stream.wait_stream(cur)          # the previous step no longer reads W, X
+        arrived = []
+        with torch.cuda.stream(copy_stream):
+            W.copy_(Wh, non_blocking=True)
+            for c in range(n_chunks):
+                a, b = bounds[c], bounds[c + 1]
+                X[a:b].copy_(Xh[a:b], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(copy_stream)
+                arrived.append(ev)
+        for c in range(n_chunks):
+            a, b = bounds[c], bounds[c + 1]
+            cur.wait_event(arrived[c])
+            z.hessian_accumulate(X[a:b], H[a:b], alpha=2.0, beta=0.0, workspace=h_ws)
+        out = z.prune_layers(W, H, g, shape.damp_frac, levels, workspace=p_ws, out=out)
         for k, v in host_out.items():
             v.copy_(out[k], non_blocking=True)
 
