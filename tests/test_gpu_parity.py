@@ -172,6 +172,26 @@ def test_neuron_path_is_deterministic(neuron_path):
     assert torch.equal(a["W_snap"], b["W_snap"])
 
 
+@pytest.mark.parametrize("groups", ["1", "3", "8"])
+def test_layer_groups_do_not_change_the_result(groups, monkeypatch):
+    """Layers are independent problems: how many groups of them run on internal streams must not
+    change a single bit of any output."""
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=320, d_row=48, d_latent=80,
+                   n_tokens=1280, n_layers=9, levels=(256, 100, 0))
+    W, X = wl.make_layers(sh, "cpu")
+    H = torch.stack([oracle_h32(X[l]) for l in range(9)]).cuda()
+    monkeypatch.delenv("ZIPLM_LAYER_GROUPS", raising=False)
+    ref = z.prune_layers(W.cuda(), H, 1, 0.01, [256, 100, 0])
+    torch.cuda.synchronize()
+    monkeypatch.setenv("ZIPLM_LAYER_GROUPS", groups)
+    got = z.prune_layers(W.cuda(), H, 1, 0.01, [256, 100, 0])
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(got["layer_status"]) == 0
+    for k in ("order", "W_snap", "loss", "base_loss", "saliency"):
+        assert torch.equal(ref[k], got[k]), k
+
+
 def test_workspace_is_not_assumed_clean(neuron_path):
     """Poison the workspace with NaN bit patterns: values of unused slots never feed live ones."""
     z = zb()
