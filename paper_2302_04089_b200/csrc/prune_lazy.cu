@@ -137,20 +137,22 @@ __device__ __forceinline__ Cand bcast_cand(const Cand& c, int src_lane) {
     return o;
 }
 
-// Best candidate of a warp (every lane returns it).  A cheap fp32 quotient orders the lanes; only
-// the lanes within 1e-5 of the fp32 minimum (almost always a single one) go through the exact
-// float64 comparison, so the common case costs six 32-bit shuffles instead of five rounds of
-// 64-bit exchanges.
 // fp32 quotient that orders candidates coarsely: +inf for "none", -inf for an invalid entry.
 __device__ __forceinline__ float cand_quotient(const Cand& c) {
     if (c.pos < 0) return INFINITY;
     return cand_valid(c) ? __fdividef((float)c.q, (float)c.a) : -INFINITY;
 }
 
+// Best candidate of a warp (every lane returns it).  The cheap fp32 quotient r orders the lanes;
+// only the lanes within 1e-5 of the fp32 minimum (almost always a single one) go through the exact
+// float64 comparison, so the common case costs one reduction and six 32-bit shuffles instead of
+// five rounds of 64-bit exchanges.
 __device__ __forceinline__ Cand warp_best(const Cand& mine, float r) {
-    float rmin = r;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) rmin = fminf(rmin, __shfl_xor_sync(0xffffffffu, rmin, off));
+    // warp minimum in one reduction instruction, on keys that order like the floats they encode
+    const unsigned bits = __float_as_uint(r);
+    const unsigned key = bits ^ ((bits >> 31) ? 0xffffffffu : 0x80000000u);
+    const unsigned kmin = __reduce_min_sync(0xffffffffu, key);
+    const float rmin = __uint_as_float(kmin ^ ((kmin >> 31) ? 0x80000000u : 0xffffffffu));
     const bool near_min = mine.pos >= 0 && (r == rmin || r <= rmin + fabsf(rmin) * 1e-5f);
     unsigned mask = __ballot_sync(0xffffffffu, near_min);
     Cand best;
