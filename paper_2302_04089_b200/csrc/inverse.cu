@@ -263,17 +263,15 @@ __device__ __forceinline__ void task_krange(const GemmTask& t, int ti, int tj, i
 // One CTA per 128 x 64 macro tile (two tiles high); blockIdx.x runs over the macro tiles of the
 // task (those that reach the lower triangle when lower_only), blockIdx.y over the layers.
 template <bool TA, bool TB>
-__global__ void __launch_bounds__(GT, 2) k_dgemm_tiles(GemmTask t, int dp) {
-    extern __shared__ __align__(16) double smem[];
-    const int l = blockIdx.y;
+__device__ __forceinline__ void dgemm_task(const GemmTask& t, int dp, int bx, int l, double* smem) {
     const int mmt = (t.mt + 1) / 2;
     // macro tiles with the longest k range come first, so that the last wave is the lightest
     int I, J;
-    if (t.lower_only) lower_macro_index(blockIdx.x, t.mt, I, J);
-    else if (t.kmode == 1) { J = t.nt - 1 - blockIdx.x / mmt; I = blockIdx.x % mmt; }
-    else if (t.kmode == 3) { J = blockIdx.x / mmt; I = blockIdx.x % mmt; }
-    else if (t.kmode == 2) { I = mmt - 1 - blockIdx.x / t.nt; J = blockIdx.x % t.nt; }
-    else { I = blockIdx.x / t.nt; J = blockIdx.x % t.nt; }
+    if (t.lower_only) lower_macro_index(bx, t.mt, I, J);
+    else if (t.kmode == 1) { J = t.nt - 1 - bx / mmt; I = bx % mmt; }
+    else if (t.kmode == 3) { J = bx / mmt; I = bx % mmt; }
+    else if (t.kmode == 2) { I = mmt - 1 - bx / t.nt; J = bx % t.nt; }
+    else { I = bx / t.nt; J = bx % t.nt; }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ti = 2 * I + (warp >> 2), tj = J;                          // this warp's tile
     const bool mine = ti < t.mt && (!t.lower_only || ti >= tj);
@@ -309,6 +307,21 @@ __global__ void __launch_bounds__(GT, 2) k_dgemm_tiles(GemmTask t, int dp) {
             if (t.beta) { const double2 c = *o; v.x += c.x; v.y += c.y; }
             *o = v;
         }
+}
+
+template <bool TA, bool TB>
+__global__ void __launch_bounds__(GT, 2) k_dgemm_tiles(GemmTask t, int dp) {
+    extern __shared__ __align__(16) double smem[];
+    dgemm_task<TA, TB>(t, dp, blockIdx.x, blockIdx.y, smem);
+}
+
+// Two independent products in one launch: the first n1 CTAs of a layer run t1 (A B^T form), the
+// rest t2 (A B form).  Used for A22 -= F21 F21^T and scratch = F21 M11, which both depend on F21
+// only: one launch fills the other's last wave.
+__global__ void __launch_bounds__(GT, 2) k_dgemm_pair(GemmTask t1, int n1, GemmTask t2, int dp) {
+    extern __shared__ __align__(16) double smem[];
+    if ((int)blockIdx.x < n1) dgemm_task<false, true>(t1, dp, blockIdx.x, blockIdx.y, smem);
+    else dgemm_task<false, false>(t2, dp, blockIdx.x - n1, blockIdx.y, smem);
 }
 
 // ---- base case of the recursion: a range of up to kSmallMax tiles, one CTA per layer ----------
@@ -698,10 +711,25 @@ struct InvCtx {
     cudaStream_t st;
 };
 
+int task_ctas(const GemmTask& t) {
+    const int mm = (t.mt + 1) / 2;                           // macro tiles: mm x t.nt
+    return t.lower_only ? lower_macro_count(t.mt) : mm * t.nt;
+}
+
+ziplm_status launch_pair(const InvCtx& c, const GemmTask& t1, const GemmTask& t2) {
+    const int n1 = task_ctas(t1), n2 = task_ctas(t2);
+    static const cudaError_t attr = cudaFuncSetAttribute(
+        k_dgemm_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
+    if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
+    PhaseScope ps(PH_INV_PRODUCTS, c.st);
+    k_dgemm_pair<<<dim3(n1 + n2, c.L), GT, kProductSmemBytes, c.st>>>(t1, n1, t2, c.dp);
+    ZIPLM_CHECK_LAUNCH();
+    return ZIPLM_OK;
+}
+
 template <bool TA, bool TB>
 ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
-    const int mm = (t.mt + 1) / 2;                           // macro tiles: mm x t.nt
-    const int ctas = t.lower_only ? lower_macro_count(t.mt) : mm * t.nt;
+    const int ctas = task_ctas(t);
     if (ctas <= 0 || t.kt <= 0) return ZIPLM_OK;
     static const cudaError_t attr = cudaFuncSetAttribute(
         k_dgemm_tiles<TA, TB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
@@ -733,13 +761,15 @@ ziplm_status factor_range(const InvCtx& c, int lo, int hi) {
     // F21 = A21 M11^T   (M11 lower triangular: opB(k,j) = M11[j,k] vanishes for k > j)
     t = GemmTask{c.A, mid, lo, c.M, lo, lo, c.F, mid, lo, n2, n1, n1, 1, 0, 1.0, 0};
     if ((s = launch_gemm<false, true>(c, t)) != ZIPLM_OK) return s;
-    // A22 -= F21 F21^T  (lower tiles)
-    t = GemmTask{c.F, mid, lo, c.F, mid, lo, c.A, mid, mid, n2, n2, n1, 0, 1, -1.0, 1};
-    if ((s = launch_gemm<false, true>(c, t)) != ZIPLM_OK) return s;
+    // A22 -= F21 F21^T  (lower tiles), and in the same launch
+    // scratch (the dead A21 block) = F21 M11   (M11 lower: opB(k,j) vanishes for k < j):
+    // its operands are final here and only the M21 product below reads it
+    {
+        const GemmTask syrk{c.F, mid, lo, c.F, mid, lo, c.A, mid, mid, n2, n2, n1, 0, 1, -1.0, 1};
+        const GemmTask scr{c.F, mid, lo, c.M, lo, lo, c.A, mid, lo, n2, n1, n1, 3, 0, 1.0, 0};
+        if ((s = launch_pair(c, syrk, scr)) != ZIPLM_OK) return s;
+    }
     if ((s = factor_range(c, mid, hi)) != ZIPLM_OK) return s;
-    // scratch (the dead A21 block) = F21 M11   (M11 lower: opB(k,j) vanishes for k < j)
-    t = GemmTask{c.F, mid, lo, c.M, lo, lo, c.A, mid, lo, n2, n1, n1, 3, 0, 1.0, 0};
-    if ((s = launch_gemm<false, false>(c, t)) != ZIPLM_OK) return s;
     // M21 = -M22 scratch  (M22 lower: opA(i,k) vanishes for k > i)
     t = GemmTask{c.M, mid, mid, c.A, mid, lo, c.M, mid, lo, n2, n1, n2, 2, 0, -1.0, 0};
     return launch_gemm<false, false>(c, t);
