@@ -877,6 +877,15 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
             ZIPLM_CHECK_LAUNCH();
         }
         const int n_new = n - nsteps;
+        // The update of W goes first: measured, the step is 2 ms shorter than with the wide update
+        // of H^-1 and Q in front (the next steps kernel then follows the kernel with the longer,
+        // finer-grained tail).
+        if (n_new > 0) {
+            PhaseScope ps(PH_LAZY_UPDATE_W, st);
+            k_lazy_update_w<<<dim3((n_new + 63) / 64, (rp + 255) / 256, L), 256, 0, st>>>(
+                n_new, nsteps, d, rp, w.Wt[cur], w.Wt[nxt], w.src, w.U, w.C);
+            ZIPLM_CHECK_LAUNCH();
+        }
         if (n_new > 1 && use_tc) {
             PhaseScope ps(PH_LAZY_UPDATE_AQ, st);
             s = run_lazy_update_aq_tc(map, L, n_new, nsteps, d, w.A[cur], w.Q[cur], w.A[nxt], w.Q[nxt],
@@ -890,12 +899,6 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
                     n_new, nsteps, d, w.A[cur], w.Q[cur], w.A[nxt], w.Q[nxt], w.src, w.U, w.Z);
                 ZIPLM_CHECK_LAUNCH();
             }
-        }
-        if (n_new > 0) {
-            PhaseScope ps(PH_LAZY_UPDATE_W, st);
-            k_lazy_update_w<<<dim3((n_new + 63) / 64, (rp + 255) / 256, L), 256, 0, st>>>(
-                n_new, nsteps, d, rp, w.Wt[cur], w.Wt[nxt], w.src, w.U, w.C);
-            ZIPLM_CHECK_LAUNCH();
         }
         cur = nxt;
         n = n_new;
