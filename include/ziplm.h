@@ -79,6 +79,39 @@ ziplm_status ziplm_hessian_accumulate(float* H, const void* X, ziplm_dtype x_dty
                                       void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Calibration Hessian from token-major activations, batch by batch (caption of Algorithm 1:
+ * H = 2 X X^T; Sec. 3.1: X are the layer inputs collected on calibration data, which a forward
+ * pass emits one token per row).
+ *
+ *   H[l] = beta * H[l] + alpha * A[l]^T A[l]        for l = 0 .. L-1
+ *
+ * A[l] is the n_tokens x d matrix whose rows are the layer's input vectors, i.e. A[l] = X[l]^T in
+ * the paper's notation, so the result is the same matrix ziplm_hessian_accumulate computes from
+ * X[l].  Calling it once per calibration batch with beta = 1 (beta = 0 on the first batch, or on a
+ * zeroed H) builds the Hessian of the whole calibration set without ever holding all activations.
+ * Arithmetic and accuracy are those of ziplm_hessian_accumulate: a pre-pass brings the batch into
+ * the token-contiguous layout (for fp32 together with the TF32 split) and the same tensor-core
+ * product kernel runs on it.
+ *
+ *   H          dev, [L, d, d] fp32, in/out; full symmetric matrix on return
+ *   A          dev, [L, n_tokens, lda] of a_dtype, feature index contiguous; only the first d
+ *              entries of each row are read; not modified.  Aligned to its element size.
+ *   lda        row pitch of A in elements, >= d
+ *   workspace  dev scratch of at least ziplm_hessian_tokens_workspace_bytes(...) bytes, 256-byte
+ *              aligned; may be NULL when that size is 0
+ *
+ * Errors: ZIPLM_ERR_INVALID_ARG for L, d < 1, n_tokens < 0, lda < d, a NULL or misaligned
+ * pointer or beta outside {0, 1}; ZIPLM_ERR_WORKSPACE; ZIPLM_ERR_CUDA.
+ * n_tokens = 0 scales H by beta and returns.
+ */
+size_t ziplm_hessian_tokens_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype a_dtype);
+
+ziplm_status ziplm_hessian_accumulate_tokens(float* H, const void* A, ziplm_dtype a_dtype, int L,
+                                             int d, long long n_tokens, long long lda, float alpha,
+                                             float beta, void* workspace, size_t workspace_bytes,
+                                             void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Damped inverse (caption of Algorithm 1: H^-1 = (2 X X^T + lambda I)^-1).
  *
  *   lambda[l] = damp_frac * mean(diag H[l]);   Hinv[l] = (H[l] + lambda[l] I)^-1

@@ -50,6 +50,21 @@ def hessian(X, alpha: float = 2.0) -> np.ndarray:
     return alpha * (X @ X.T)
 
 
+def hessian_from_token_batches(batches, alpha: float = 2.0) -> np.ndarray:
+    """H = alpha * sum over all calibration tokens x of x x^T (Algorithm 1 caption with X written
+    column by column: X X^T is the sum of the outer products of its columns).  ``batches`` is a
+    sequence of token-major matrices [n_b, d_col], one token per row, as a forward pass emits the
+    layer inputs; the result does not depend on how the tokens are cut into batches."""
+    H = None
+    for A in batches:
+        A = as_f64(A)
+        part = np.zeros((A.shape[1], A.shape[1]))
+        for x in A:
+            part += np.outer(x, x)
+        H = part if H is None else H + part
+    return alpha * H
+
+
 def damped(H, damp_frac: float):
     """(H + lambda I, lambda) with lambda = damp_frac * mean(diag H) (Algorithm 1 caption)."""
     H = as_f64(H)

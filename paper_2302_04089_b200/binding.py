@@ -61,6 +61,11 @@ def load_library() -> ctypes.CDLL:
     lib.ziplm_hessian_accumulate.restype = c_int
     lib.ziplm_hessian_accumulate.argtypes = [vp, vp, c_int, c_int, c_int, c_ll, c_ll, c_f, c_f, vp,
                                              c_sz, vp]
+    lib.ziplm_hessian_tokens_workspace_bytes.restype = c_sz
+    lib.ziplm_hessian_tokens_workspace_bytes.argtypes = [c_int, c_int, c_ll, c_int]
+    lib.ziplm_hessian_accumulate_tokens.restype = c_int
+    lib.ziplm_hessian_accumulate_tokens.argtypes = [vp, vp, c_int, c_int, c_int, c_ll, c_ll, c_f, c_f,
+                                                    vp, c_sz, vp]
     lib.ziplm_inverse_workspace_bytes.restype = c_sz
     lib.ziplm_inverse_workspace_bytes.argtypes = [c_int, c_int]
     lib.ziplm_damped_inverse.restype = c_int
@@ -116,6 +121,10 @@ def hessian_workspace_bytes(L: int, d: int, n_tokens: int, x_dtype: int) -> int:
     return int(load_library().ziplm_hessian_workspace_bytes(L, d, n_tokens, x_dtype))
 
 
+def hessian_tokens_workspace_bytes(L: int, d: int, n_tokens: int, a_dtype: int) -> int:
+    return int(load_library().ziplm_hessian_tokens_workspace_bytes(L, d, n_tokens, a_dtype))
+
+
 def inverse_workspace_bytes(L: int, d: int) -> int:
     return int(load_library().ziplm_inverse_workspace_bytes(L, d))
 
@@ -149,6 +158,37 @@ def hessian_accumulate(X: torch.Tensor, H: Optional[torch.Tensor] = None, alpha:
                                           workspace.data_ptr(), workspace.numel(), _stream_ptr(X))
     if st != 0:
         raise ZiplmError(st, "ziplm_hessian_accumulate")
+    return H
+
+
+def hessian_accumulate_tokens(A: torch.Tensor, H: Optional[torch.Tensor] = None, alpha: float = 2.0,
+                              beta: float = 0.0,
+                              workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """H = beta * H + alpha * A^T A per layer.  A [L, N, d] fp32 or bf16, one token per row
+    (features contiguous); the row pitch may exceed d.  See ziplm_hessian_accumulate_tokens."""
+    lib = load_library()
+    if A.dim() != 3 or not A.is_cuda or A.stride(2) != 1 and A.shape[2] > 1:
+        raise ValueError("A must be a CUDA tensor [L, N, d] with contiguous features")
+    if A.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("A must be fp32 or bf16")
+    L, N, d = A.shape
+    lda = A.stride(1) if N > 1 else d
+    if L > 1 and N > 0 and A.stride(0) != N * lda:
+        raise ValueError("layers of A must be evenly pitched")
+    dt = F32 if A.dtype == torch.float32 else BF16
+    if H is None:
+        H = torch.zeros(L, d, d, dtype=torch.float32, device=A.device)
+        beta = 0.0
+    _check(H, torch.float32, "H")
+    need = hessian_tokens_workspace_bytes(L, d, N, dt)
+    if workspace is None:
+        workspace = _workspace(need, A.device)
+    with torch.cuda.device(A.device):
+        st = lib.ziplm_hessian_accumulate_tokens(H.data_ptr(), A.data_ptr(), dt, L, d, N, lda, alpha,
+                                                 beta, workspace.data_ptr(), workspace.numel(),
+                                                 _stream_ptr(A))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_hessian_accumulate_tokens")
     return H
 
 

@@ -43,7 +43,7 @@ const char* ziplm_status_string(ziplm_status s) {
 
 size_t ziplm_hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype x_dtype) {
     if (L < 1 || d < 1 || n_tokens < 0) return 0;
-    return hessian_workspace_bytes(L, d, n_tokens, x_dtype);
+    return hessian_workspace_bytes(L, d, n_tokens, x_dtype, false);
 }
 
 ziplm_status ziplm_hessian_accumulate(float* H, const void* X, ziplm_dtype x_dtype, int L, int d,
@@ -56,13 +56,36 @@ ziplm_status ziplm_hessian_accumulate(float* H, const void* X, ziplm_dtype x_dty
     if (n_tokens > 0) {
         if (!X || !aligned(X, 16) || ((size_t)ldx * esz) % 16 != 0) return ZIPLM_ERR_INVALID_ARG;
     }
-    const size_t need = hessian_workspace_bytes(L, d, n_tokens, x_dtype);
+    const size_t need = hessian_workspace_bytes(L, d, n_tokens, x_dtype, false);
     if (need > 0 && (!workspace || !aligned(workspace, kAlign) || workspace_bytes < need))
         return ZIPLM_ERR_WORKSPACE;
     if (!have_device()) return ZIPLM_ERR_CUDA;
     PhaseScope ps(PH_HESSIAN, static_cast<cudaStream_t>(cuda_stream));
-    return run_hessian(H, X, x_dtype, L, d, n_tokens, ldx, alpha, beta, workspace, workspace_bytes,
-                       static_cast<cudaStream_t>(cuda_stream));
+    return run_hessian(H, X, x_dtype, false, L, d, n_tokens, ldx, alpha, beta, workspace,
+                       workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t ziplm_hessian_tokens_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype a_dtype) {
+    if (L < 1 || d < 1 || n_tokens < 0) return 0;
+    return hessian_workspace_bytes(L, d, n_tokens, a_dtype, true);
+}
+
+ziplm_status ziplm_hessian_accumulate_tokens(float* H, const void* A, ziplm_dtype a_dtype, int L,
+                                             int d, long long n_tokens, long long lda, float alpha,
+                                             float beta, void* workspace, size_t workspace_bytes,
+                                             void* cuda_stream) {
+    if (L < 1 || d < 1 || n_tokens < 0 || lda < d || !H) return ZIPLM_ERR_INVALID_ARG;
+    if (a_dtype != ZIPLM_F32 && a_dtype != ZIPLM_BF16) return ZIPLM_ERR_INVALID_ARG;
+    if (!(beta == 0.f || beta == 1.f) || !isfinite(alpha)) return ZIPLM_ERR_INVALID_ARG;
+    const size_t esz = (a_dtype == ZIPLM_F32) ? 4 : 2;
+    if (n_tokens > 0 && (!A || !aligned(A, esz))) return ZIPLM_ERR_INVALID_ARG;
+    const size_t need = hessian_workspace_bytes(L, d, n_tokens, a_dtype, true);
+    if (need > 0 && (!workspace || !aligned(workspace, kAlign) || workspace_bytes < need))
+        return ZIPLM_ERR_WORKSPACE;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    PhaseScope ps(PH_HESSIAN, static_cast<cudaStream_t>(cuda_stream));
+    return run_hessian(H, A, a_dtype, true, L, d, n_tokens, lda, alpha, beta, workspace,
+                       workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 size_t ziplm_inverse_workspace_bytes(int L, int d) {

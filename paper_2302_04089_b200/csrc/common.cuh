@@ -102,13 +102,15 @@ ziplm_status run_base_loss(const float* W, const float* H, int L, int r, int d, 
                            float* base_loss, cudaStream_t st);
 
 // Tensor-core route of the Hessian (hessian_tc.cu) and the route choice (hessian.cu).
-size_t hessian_tc_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt);
-ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, int L, int d, long long N,
-                            long long ldx, float alpha, float beta, void* ws, size_t ws_bytes,
-                            cudaStream_t st);
-size_t hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt);
-ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, int L, int d, long long N,
-                         long long ldx, float alpha, float beta, void* ws, size_t ws_bytes,
-                         cudaStream_t st);
+// token_major = false: X is [L, d, ldx], token index contiguous; true: X is [L, N, ldx], one
+// token per row, feature index contiguous.
+size_t hessian_tc_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt, bool token_major);
+ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_major, int L, int d,
+                            long long N, long long ldx, float alpha, float beta, void* ws,
+                            size_t ws_bytes, cudaStream_t st);
+size_t hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt, bool token_major);
+ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, bool token_major, int L, int d,
+                         long long N, long long ldx, float alpha, float beta, void* ws,
+                         size_t ws_bytes, cudaStream_t st);
 
 }  // namespace ziplm

@@ -43,7 +43,9 @@ __device__ __forceinline__ float to_f32<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-template <typename T>
+// TOK: the input is token-major, [N, ldx] per layer with the feature index contiguous; element
+// (feature i, token k) then sits at k * ldx + i and is fetched with scalar loads.
+template <typename T, bool TOK>
 __global__ void __launch_bounds__(256) k_syrk_simt(float* __restrict__ H, const T* __restrict__ X,
                                                    int d, long long N, long long ldx, float alpha,
                                                    float beta) {
@@ -53,7 +55,7 @@ __global__ void __launch_bounds__(256) k_syrk_simt(float* __restrict__ H, const 
     while (rem > ti) { rem -= ti + 1; ++ti; }
     const int tj = rem;
     const int i0 = ti * 64, j0 = tj * 64;
-    const T* Xl = X + (size_t)l * d * ldx;
+    const T* Xl = X + (size_t)l * (TOK ? (size_t)N : (size_t)d) * ldx;
     float* Hl = H + (size_t)l * d * d;
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
     float acc[4][4], tot[4][4];
@@ -66,17 +68,26 @@ __global__ void __launch_bounds__(256) k_syrk_simt(float* __restrict__ H, const 
     for (long long k0 = 0; k0 < N; k0 += BK) {
         float va[4] = {0.f, 0.f, 0.f, 0.f}, vb[4] = {0.f, 0.f, 0.f, 0.f};
         const long long k = k0 + kq;
-        if (i0 + lr < d) {
-            const T* pa = Xl + (size_t)(i0 + lr) * ldx + k;
-            if (k + 3 < N) load4<T>(pa, va);
-            else
-                for (int e = 0; e < 4; ++e) if (k + e < N) va[e] = to_f32<T>(pa[e]);
-        }
-        if (j0 + lr < d) {
-            const T* pb = Xl + (size_t)(j0 + lr) * ldx + k;
-            if (k + 3 < N) load4<T>(pb, vb);
-            else
-                for (int e = 0; e < 4; ++e) if (k + e < N) vb[e] = to_f32<T>(pb[e]);
+        if (TOK) {
+            for (int e = 0; e < 4; ++e) {
+                if (k + e >= N) break;
+                const T* pk = Xl + (size_t)(k + e) * ldx;
+                if (i0 + lr < d) va[e] = to_f32<T>(pk[i0 + lr]);
+                if (j0 + lr < d) vb[e] = to_f32<T>(pk[j0 + lr]);
+            }
+        } else {
+            if (i0 + lr < d) {
+                const T* pa = Xl + (size_t)(i0 + lr) * ldx + k;
+                if (k + 3 < N) load4<T>(pa, va);
+                else
+                    for (int e = 0; e < 4; ++e) if (k + e < N) va[e] = to_f32<T>(pa[e]);
+            }
+            if (j0 + lr < d) {
+                const T* pb = Xl + (size_t)(j0 + lr) * ldx + k;
+                if (k + 3 < N) load4<T>(pb, vb);
+                else
+                    for (int e = 0; e < 4; ++e) if (k + e < N) vb[e] = to_f32<T>(pb[e]);
+            }
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) { sA[kq + e][lr] = va[e]; sB[kq + e][lr] = vb[e]; }
@@ -126,13 +137,13 @@ bool use_tensor_cores(long long N) {
 
 }  // namespace
 
-size_t hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt) {
-    return use_tensor_cores(n_tokens) ? hessian_tc_workspace_bytes(L, d, n_tokens, dt) : 0;
+size_t hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt, bool token_major) {
+    return use_tensor_cores(n_tokens) ? hessian_tc_workspace_bytes(L, d, n_tokens, dt, token_major) : 0;
 }
 
-ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, int L, int d, long long N,
-                         long long ldx, float alpha, float beta, void* ws, size_t ws_bytes,
-                         cudaStream_t st) {
+ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, bool token_major, int L, int d,
+                         long long N, long long ldx, float alpha, float beta, void* ws,
+                         size_t ws_bytes, cudaStream_t st) {
     if (N == 0) {
         const size_t count = (size_t)L * d * d;
         if (beta != 1.f) {
@@ -142,14 +153,19 @@ ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, int L, int d, 
         return ZIPLM_OK;
     }
     if (use_tensor_cores(N))
-        return run_hessian_tc(H, X, dt, L, d, N, ldx, alpha, beta, ws, ws_bytes, st);
+        return run_hessian_tc(H, X, dt, token_major, L, d, N, ldx, alpha, beta, ws, ws_bytes, st);
     const int T = (d + 63) / 64;
     const dim3 grid(T * (T + 1) / 2, L);
-    if (dt == ZIPLM_F32)
-        k_syrk_simt<float><<<grid, 256, 0, st>>>(H, static_cast<const float*>(X), d, N, ldx, alpha, beta);
+    const float* Xf = static_cast<const float*>(X);
+    const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
+    if (dt == ZIPLM_F32 && !token_major)
+        k_syrk_simt<float, false><<<grid, 256, 0, st>>>(H, Xf, d, N, ldx, alpha, beta);
+    else if (dt == ZIPLM_F32)
+        k_syrk_simt<float, true><<<grid, 256, 0, st>>>(H, Xf, d, N, ldx, alpha, beta);
+    else if (!token_major)
+        k_syrk_simt<__nv_bfloat16, false><<<grid, 256, 0, st>>>(H, Xb, d, N, ldx, alpha, beta);
     else
-        k_syrk_simt<__nv_bfloat16><<<grid, 256, 0, st>>>(H, static_cast<const __nv_bfloat16*>(X), d, N,
-                                                       ldx, alpha, beta);
+        k_syrk_simt<__nv_bfloat16, true><<<grid, 256, 0, st>>>(H, Xb, d, N, ldx, alpha, beta);
     ZIPLM_CHECK_LAUNCH();
     return ZIPLM_OK;
 }

@@ -263,6 +263,46 @@ __global__ void __launch_bounds__(256) k_split_tf32(const float* __restrict__ X,
     *reinterpret_cast<float4*>(lo + row * (size_t)np + k) = make_float4(w[0], w[1], w[2], w[3]);
 }
 
+// Token-major input (one calibration token per row, as a forward pass emits activations):
+// A is [layers, N, lda] with the feature index contiguous.  A 32 x 32 tile goes through shared
+// memory, so the reads run along features and the writes along tokens, both coalesced; the output
+// is the K-major [layers * d, np] matrix the product kernel loads.  SPLIT writes the TF32 parts
+// X_hi / X_lo of an fp32 input directly (same values as k_split_tf32); otherwise the elements
+// are moved as raw bits (T = uint16_t for bf16).
+template <typename T, bool SPLIT>
+__global__ void __launch_bounds__(256) k_tokens_to_kmajor(const T* __restrict__ A, long long lda,
+                                                          long long N, int d, long long np,
+                                                          T* __restrict__ hi, T* __restrict__ lo) {
+    __shared__ T tile[32][33];
+    const int l = blockIdx.z;
+    const long long t0 = (long long)blockIdx.x * 32;
+    const int f0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const T* Al = A + (size_t)l * (size_t)N * (size_t)lda;
+#pragma unroll
+    for (int r = ty; r < 32; r += 8) {
+        const long long t = t0 + r;
+        const int f = f0 + tx;
+        tile[r][tx] = (t < N && f < d) ? Al[(size_t)t * (size_t)lda + f] : T(0);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = ty; r < 32; r += 8) {
+        const int f = f0 + r;
+        const long long t = t0 + tx;
+        if (f >= d || t >= np) continue;
+        const size_t o = ((size_t)l * d + f) * (size_t)np + (size_t)t;
+        const T v = tile[tx][r];
+        if constexpr (SPLIT) {
+            const float h = __uint_as_float(__float_as_uint(v) & 0xffffe000u);
+            hi[o] = h;
+            lo[o] = v - h;
+        } else {
+            hi[o] = v;
+        }
+    }
+}
+
 // 3-D map over [layers, rows, K] with box {128 bytes of K, 128 rows, 1 layer}, 128-byte swizzle,
 // zero fill outside the tensor (ragged d and ragged token counts contribute zeros).
 bool make_map(CUtensorMap* m, const void* base, bool f32, long long K, int rows, int layers,
@@ -284,6 +324,16 @@ bool make_map(CUtensorMap* m, const void* base, bool f32, long long K, int rows,
 constexpr size_t kSplitCapBytes = (size_t)8 << 30;   // bound on the hi/lo scratch of one chunk
 
 long long padded_tokens(long long N) { return (N + 3) / 4 * 4; }
+long long padded_tokens_bf16(long long N) { return (N + 7) / 8 * 8; }   // 16-byte row pitch
+
+// Layers per chunk of the K-major bf16 copy of a token-major input.
+int transpose_chunk_layers(int L, int d, long long N) {
+    const size_t per_layer = (size_t)d * (size_t)padded_tokens_bf16(N) * 2;
+    size_t lc = kSplitCapBytes / (per_layer ? per_layer : 1);
+    if (lc < 1) lc = 1;
+    if (lc > 65535) lc = 65535;
+    return (int)(lc < (size_t)L ? lc : (size_t)L);
+}
 
 int split_chunk_layers(int L, int d, long long N) {
     const size_t per_layer = 2 * (size_t)d * (size_t)padded_tokens(N) * 4;
@@ -294,19 +344,22 @@ int split_chunk_layers(int L, int d, long long N) {
 
 }  // namespace
 
-size_t hessian_tc_workspace_bytes(int L, int d, long long N, ziplm_dtype dt) {
+size_t hessian_tc_workspace_bytes(int L, int d, long long N, ziplm_dtype dt, bool token_major) {
     size_t b = kAlign;   // error word
     if (dt == ZIPLM_F32) {
         const int lc = split_chunk_layers(L, d, N);
         b += 2 * align_up((size_t)lc * d * (size_t)padded_tokens(N) * 4);
+    } else if (token_major) {
+        const int lc = transpose_chunk_layers(L, d, N);
+        b += align_up((size_t)lc * d * (size_t)padded_tokens_bf16(N) * 2);
     }
     return b;
 }
 
-ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, int L, int d, long long N,
-                            long long ldx, float alpha, float beta, void* ws, size_t ws_bytes,
-                            cudaStream_t st) {
-    if (ws_bytes < hessian_tc_workspace_bytes(L, d, N, dt)) return ZIPLM_ERR_WORKSPACE;
+ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_major, int L, int d,
+                            long long N, long long ldx, float alpha, float beta, void* ws,
+                            size_t ws_bytes, cudaStream_t st) {
+    if (ws_bytes < hessian_tc_workspace_bytes(L, d, N, dt, token_major)) return ZIPLM_ERR_WORKSPACE;
     const bool f32 = (dt == ZIPLM_F32);
     Carver c(ws);
     int* err_word = c.take<int>(1);
@@ -331,19 +384,51 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, int L, int 
         for (int l0 = 0; l0 < L; l0 += lc) {
             const int ln = (L - l0 < lc) ? (L - l0) : lc;
             const size_t rows = (size_t)ln * d;
-            const float* Xc = static_cast<const float*>(X) + (size_t)l0 * d * ldx;
-            // grid.y is limited to 65535 rows per launch
-            for (size_t r0 = 0; r0 < rows; r0 += 65535) {
-                const size_t rn = rows - r0 < 65535 ? rows - r0 : 65535;
-                k_split_tf32<<<dim3((unsigned)((np / 4 + 255) / 256), (unsigned)rn), 256, 0, st>>>(
-                    Xc + r0 * ldx, ldx, N, np, rn, hi + r0 * np, lo + r0 * np);
-                ZIPLM_CHECK_LAUNCH();
+            if (token_major) {
+                const float* Ac = static_cast<const float*>(X) + (size_t)l0 * (size_t)N * ldx;
+                // grid.z is limited to 65535 layers per launch
+                for (int z0 = 0; z0 < ln; z0 += 65535) {
+                    const int zn = ln - z0 < 65535 ? ln - z0 : 65535;
+                    k_tokens_to_kmajor<float, true>
+                        <<<dim3((unsigned)((np + 31) / 32), (unsigned)((d + 31) / 32), (unsigned)zn), 256, 0,
+                           st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, np, hi + (size_t)z0 * d * np,
+                                 lo + (size_t)z0 * d * np);
+                    ZIPLM_CHECK_LAUNCH();
+                }
+            } else {
+                const float* Xc = static_cast<const float*>(X) + (size_t)l0 * d * ldx;
+                // grid.y is limited to 65535 rows per launch
+                for (size_t r0 = 0; r0 < rows; r0 += 65535) {
+                    const size_t rn = rows - r0 < 65535 ? rows - r0 : 65535;
+                    k_split_tf32<<<dim3((unsigned)((np / 4 + 255) / 256), (unsigned)rn), 256, 0, st>>>(
+                        Xc + r0 * ldx, ldx, N, np, rn, hi + r0 * np, lo + r0 * np);
+                    ZIPLM_CHECK_LAUNCH();
+                }
             }
             CUtensorMap mh, ml;
             if (!make_map(&mh, hi, true, N, d, ln, np) || !make_map(&ml, lo, true, N, d, ln, np))
                 return ZIPLM_ERR_CUDA;
             k_syrk_tc<true><<<dim3(n_tiles, ln), THREADS, smem_tf32, st>>>(mh, ml, H, d, num_kb, alpha, beta,
                                                                       l0, err_word);
+            ZIPLM_CHECK_LAUNCH();
+        }
+    } else if (token_major) {
+        // K-major bf16 copy of a chunk of layers, then the same product kernel
+        const long long np = padded_tokens_bf16(N);
+        const int lc = transpose_chunk_layers(L, d, N);
+        uint16_t* xt = c.take<uint16_t>((size_t)lc * d * np);
+        const int num_kb = (int)((N + Cfg<false>::BK - 1) / Cfg<false>::BK);
+        for (int l0 = 0; l0 < L; l0 += lc) {
+            const int ln = (L - l0 < lc) ? (L - l0) : lc;
+            const uint16_t* Ac = static_cast<const uint16_t*>(X) + (size_t)l0 * (size_t)N * ldx;
+            k_tokens_to_kmajor<uint16_t, false>
+                <<<dim3((unsigned)((np + 31) / 32), (unsigned)((d + 31) / 32), (unsigned)ln), 256, 0, st>>>(
+                    Ac, ldx, N, d, np, xt, nullptr);
+            ZIPLM_CHECK_LAUNCH();
+            CUtensorMap mx;
+            if (!make_map(&mx, xt, false, N, d, ln, np)) return ZIPLM_ERR_CUDA;
+            k_syrk_tc<false><<<dim3(n_tiles, ln), THREADS, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
+                                                                       l0, err_word);
             ZIPLM_CHECK_LAUNCH();
         }
     } else {

@@ -766,7 +766,7 @@ LazyWs carve_lazy(void* ws, int L, int r, int d) {
     w.lam = c.take<double>((size_t)L);
     w.base_acc = c.take<double>((size_t)L);
     const size_t inv = inverse_workspace_bytes(L, d);
-    const size_t gram = hessian_tc_workspace_bytes(L, d, w.rp, ZIPLM_F32);
+    const size_t gram = hessian_tc_workspace_bytes(L, d, w.rp, ZIPLM_F32, false);
     w.aux_bytes = inv > gram ? inv : gram;
     w.aux = c.take<char>(w.aux_bytes);
     w.total = c.off;
@@ -806,7 +806,7 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
                                                            w.state);
         ZIPLM_CHECK_LAUNCH();
         // Q = W^T W: the symmetric product kernel of the Hessian with X = W^T (K = d_row)
-        ziplm_status g = run_hessian_tc(w.Q[0], w.Wt[0], ZIPLM_F32, L, d, rp, rp, 1.0f, 0.0f, w.aux,
+        ziplm_status g = run_hessian_tc(w.Q[0], w.Wt[0], ZIPLM_F32, false, L, d, rp, rp, 1.0f, 0.0f, w.aux,
                                         w.aux_bytes, st);
         if (g != ZIPLM_OK) return g;
         if (base_loss) {

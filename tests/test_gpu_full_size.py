@@ -190,3 +190,65 @@ def test_c5_gpt2_bf16_activations_both_shapes():
         check_late_step(Wl, H_or[6], mlp, out, 6, t)
     for slot in (1, 8, 9):                 # levels 2457, 307, 0
         check_level(Wl, H_or[6], mlp, out, 6, slot)
+
+
+def stream_token_major(shape, n_batches):
+    """The Hessian of all layers from token-major batches (one token per row, the layout a forward
+    pass emits), accumulated batch by batch with beta = 1.  Returns (X [L, d, N] on the GPU, H)."""
+    z = zb()
+    L, N, d = shape.n_layers, shape.n_tokens, shape.d_col
+    X = torch.stack([wl.make_activations(shape, l, "cuda") for l in range(L)])
+    H = torch.empty(L, d, d, device="cuda")
+    step = N // n_batches
+    ws = None
+    for b in range(n_batches):
+        A = X[:, :, b * step:(b + 1) * step].transpose(1, 2).contiguous()      # [L, step, d]
+        if ws is None:
+            dt = 0 if A.dtype == torch.float32 else 1
+            ws = torch.empty(z.hessian_tokens_workspace_bytes(L, d, step, dt) + 256,
+                             dtype=torch.uint8, device="cuda")
+        z.hessian_accumulate_tokens(A, H, beta=0.0 if b == 0 else 1.0, workspace=ws)
+        del A
+    torch.cuda.synchronize()
+    return X, H
+
+
+def test_paper_database_grid_from_streamed_token_major_batches():
+    """The per-layer database as the paper builds it (Sec. 3.2): FFN sizes 0.9^i * 3072 down to
+    about 99 % sparsity plus the dropped module, the Hessian accumulated batch by batch from
+    token-major fp32 activations; and the same accumulation for bf16 activations of the GPT-2
+    attention shape (131072 tokens in 16 batches)."""
+    z = zb()
+    base = wl.CONFIGS["c3_bert_base_fc2"][0]
+    shape = wl.scaled(base, levels=wl.paper_level_grid(base.n_groups, 1))
+    assert len(shape.levels) == 43
+    X, H = stream_token_major(shape, 8)
+    l = 5
+    Ho = zo.hessian(X[l])
+    scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
+    err = np.max(np.abs(H[l].cpu().double().numpy() - Ho) / scale)
+    assert err < hessian_tol("f32"), err
+    # eight batches and one pass differ only by the rounding of seven more fp32 additions
+    H1 = z.hessian_accumulate(X[l:l + 1])
+    assert torch.allclose(H[l], H1[0], rtol=0, atol=4e-6 * float(H1[0].diagonal().max()))
+    del X, H1
+    H32 = Ho.astype(np.float32)
+    H[l].copy_(torch.from_numpy(H32))
+    W = torch.stack([wl.make_weight(shape, k) for k in range(shape.n_layers)]).cuda()
+    out = z.prune_layers(W, H, 1, shape.damp_frac, list(shape.levels))
+    torch.cuda.synchronize()
+    generic_properties(shape, out)
+    Wl = W[l].cpu().numpy()
+    lockstep_head(Wl, H32, shape, out, l, 24)
+    for slot in (0, 7, 21, 41, 42):          # sizes 2764, 1322, 302, 36, 0
+        check_level(Wl, H32, shape, out, l, slot)
+    del W, out, H
+    torch.cuda.empty_cache()
+
+    attn = wl.CONFIGS["c5_gpt2"][0]
+    X, H = stream_token_major(attn, 16)
+    for l in (0, 11):
+        Ho = zo.hessian(X[l])
+        scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
+        err = np.max(np.abs(H[l].cpu().double().numpy() - Ho) / scale)
+        assert err < hessian_tol("bf16"), err

@@ -72,6 +72,83 @@ def test_hessian_zero_tokens_and_bad_args():
         z.hessian_accumulate(torch.zeros(1, 8, 8, device="cuda"), H.clone(), beta=0.5)
 
 
+# ------------------------------------------------------------------ Hessian from token-major batches
+def token_major_case(dtype, d, N, lda, L=2):
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=d, d_latent=32, n_tokens=N,
+                   n_layers=L, x_dtype=dtype)
+    _, X = wl.make_layers(sh, "cpu")                      # [L, d, N]
+    A = torch.zeros(L, N, lda, dtype=X.dtype)
+    A[:, :, :d] = X.transpose(1, 2)
+    if lda > d:
+        A[:, :, d:] = 7.0                                  # pitch padding must never be read
+    return X, A
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,N,lda", [(64, 256, 64), (200, 1000, 208), (130, 613, 131), (96, 8, 96),
+                                     (33, 31, 40), (257, 4099, 257)])
+def test_hessian_from_token_major_activations_matches_oracle(dtype, d, N, lda):
+    z = zb()
+    X, A = token_major_case(dtype, d, N, lda)
+    Ad = A.cuda()[:, :, :d]
+    H = z.hessian_accumulate_tokens(Ad)
+    torch.cuda.synchronize()
+    for l in range(2):
+        Ho = zo.hessian(X[l])
+        scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
+        err = np.max(np.abs(H[l].cpu().double().numpy() - Ho) / scale)
+        assert err < 2e-6, err
+        assert torch.equal(H[l], H[l].T)
+    # same numbers, to the bit, as the token-contiguous entry point where that one accepts the
+    # layout (16-byte row pitch) and both take the same route
+    if (N * X.element_size()) % 16 == 0:
+        assert torch.equal(H, z.hessian_accumulate(X.cuda()))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_hessian_streamed_batch_by_batch(dtype):
+    """beta = 1 over ragged calibration batches (one of them shorter than a K block, one empty)
+    against the oracle's sum of outer products over all tokens."""
+    z = zb()
+    d, N = 160, 1500
+    X, A = token_major_case(dtype, d, N, d, L=3)
+    cuts = [0, 512, 512, 531, 1100, 1500]
+    Ad = A.cuda()
+    H = torch.full((3, d, d), float("nan"), device="cuda")
+    for b in range(len(cuts) - 1):
+        part = Ad[:, cuts[b]:cuts[b + 1], :].contiguous()
+        z.hessian_accumulate_tokens(part, H, beta=0.0 if b == 0 else 1.0)
+    torch.cuda.synchronize()
+    for l in range(3):
+        Ho = zo.hessian_from_token_batches([A[l, cuts[b]:cuts[b + 1]] for b in range(len(cuts) - 1)]) \
+            if l == 0 else zo.hessian(X[l])
+        scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
+        err = np.max(np.abs(H[l].cpu().double().numpy() - Ho) / scale)
+        assert err < 2e-6, err
+
+
+def test_hessian_tokens_bad_args():
+    z = zb()
+    H = torch.ones(1, 8, 8, device="cuda")
+    A0 = torch.zeros(1, 0, 8, device="cuda")
+    assert torch.equal(z.hessian_accumulate_tokens(A0, H.clone(), beta=1.0), H)
+    assert torch.count_nonzero(z.hessian_accumulate_tokens(A0, H.clone(), beta=0.0)) == 0
+    with pytest.raises(z.ZiplmError):
+        z.hessian_accumulate_tokens(torch.zeros(1, 4, 8, device="cuda"), H.clone(), beta=0.5)
+    lib = z.load_library()
+    a = torch.zeros(4, 8, device="cuda")
+    ws = torch.empty(z.hessian_tokens_workspace_bytes(1, 8, 4, 0) + 256, dtype=torch.uint8, device="cuda")
+    # row pitch smaller than the feature count
+    assert lib.ziplm_hessian_accumulate_tokens(H.data_ptr(), a.data_ptr(), 0, 1, 8, 4, 7, 2.0, 0.0,
+                                               ws.data_ptr(), ws.numel(), None) == z.Status.ERR_INVALID_ARG
+    # workspace too small on the tensor-core route
+    need = z.hessian_tokens_workspace_bytes(1, 8, 64, 0)
+    assert need > 0
+    a64 = torch.zeros(64, 8, device="cuda")
+    assert lib.ziplm_hessian_accumulate_tokens(H.data_ptr(), a64.data_ptr(), 0, 1, 8, 64, 8, 2.0, 0.0,
+                                               ws.data_ptr(), need - 256, None) == z.Status.ERR_WORKSPACE
+
+
 # ------------------------------------------------------------------ damped inverse (a2, a3)
 @pytest.mark.parametrize("d,L", [(64, 1), (100, 2), (256, 3), (448, 1), (827, 1), (1100, 2)])
 def test_damped_inverse_matches_oracle(d, L):

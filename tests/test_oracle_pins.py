@@ -336,6 +336,63 @@ def test_hessian_against_naive_triple_loop_and_symmetry():
     assert np.allclose(H_lam - H, lam * np.eye(d), atol=1e-15)
 
 
+def test_token_batch_hessian_is_the_hessian_of_the_layer_error():
+    """Token-major, batch-by-batch form: independent of the cut into batches, equal entry by
+    entry to a plain triple loop, equal to the feature-major form on the transposed matrix, and
+    -- what makes it the Hessian of Eq. 1 -- w H w^T = 2 * sum_t (w . x_t)^2 for any row w."""
+    rng = np.random.default_rng(10)
+    d, N = 6, 11
+    A = rng.normal(size=(N, d))                      # one token per row
+    cuts = [A[:4], A[4:5], A[5:5], A[5:]]            # ragged batches, one of them empty
+    H = zo.hessian_from_token_batches(cuts)
+    naive = np.zeros((d, d))
+    for t in range(N):
+        for i in range(d):
+            for j in range(d):
+                naive[i, j] += 2.0 * A[t, i] * A[t, j]
+    assert np.allclose(H, naive, rtol=1e-13, atol=1e-14)
+    assert np.allclose(H, zo.hessian_from_token_batches([A]), rtol=1e-13, atol=1e-14)
+    assert np.allclose(H, zo.hessian(A.T), rtol=1e-13, atol=1e-14)
+    for _ in range(3):
+        w = rng.normal(size=d)
+        direct = 2.0 * sum(float(w @ A[t]) ** 2 for t in range(N))
+        assert np.isclose(w @ H @ w, direct, rtol=1e-12)
+    # a transposed operand (A A^T instead of A^T A) would not even have this shape
+    assert H.shape == (d, d)
+
+
+def test_level_grid_against_the_sizes_the_paper_prints():
+    """The database's level grid (Sec. 3.2): the FFN sizes 0.9^i * d printed in the example
+    latency table are met by the truncating grid (1814 is printed where the formula gives
+    1813.98; 33 is the step after i = 42), and heads are pruned one at a time down to none."""
+    vals = {}
+    for line in open(os.path.join(GOLD, "latency_table_sizes.txt")):
+        if line.strip() and not line.startswith("#"):
+            k, *v = line.split()
+            vals[k] = [int(x) for x in v]
+    d = vals["intermediate_sizes"][0]
+    grid = wl.ffn_size_grid(d)
+    assert len(grid) == 43 and grid[0] == d
+    assert abs(1.0 - grid[-1] / d - 0.99) < 0.003            # "until about 99 % sparsity"
+    for i in range(1, 43):
+        assert abs(grid[i] / grid[i - 1] - 0.9) < 0.02        # relative steps of 10 %
+    for size in vals["intermediate_sizes"]:
+        if size == 1814:
+            assert 1813 in grid
+        elif size == 33:
+            assert wl.ffn_size_grid(d, 43)[-1] == 33 and 33 not in grid
+        else:
+            assert size in grid, size
+    levels = wl.paper_level_grid(d, 1)
+    assert levels[-1] == 0 and d not in levels
+    assert all(a > b for a, b in zip(levels, levels[1:]))
+    assert set(levels) - {0} == set(grid) - {d}
+    G = vals["head_counts"][0]
+    heads = wl.paper_level_grid(G, 64)
+    assert heads == tuple(range(G - 1, -1, -1))
+    assert set(vals["head_counts"]) - {G} <= set(heads)
+
+
 def test_bf16_and_fp32_inputs_are_widened_exactly():
     import torch
     x = torch.tensor([[1.0, 0.333251953125, -2.5]], dtype=torch.bfloat16)

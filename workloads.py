@@ -52,6 +52,28 @@ def _even_levels(G: int, parts: int) -> Tuple[int, ...]:
     return tuple(sorted({(G * i) // parts for i in range(parts)}, reverse=True))
 
 
+def ffn_size_grid(d: int, steps: int = 42) -> Tuple[int, ...]:
+    """Intermediate sizes d * 0.9^i, i = 0 .. steps, truncated to integers (Sec. 3.2, "Runtime
+    awareness": relative steps of 10 % up to about 99 % sparsity).  Truncation is a reading: of the
+    sizes the latency-table appendix prints for d = 3072 it reproduces 1322, 302, 130 and 76
+    exactly (rounding to nearest gives 303 and 77), 1814 is printed where 0.9^5 gives 1813.98, and
+    33 is i = 43."""
+    return tuple(int(d * 0.9 ** i) for i in range(steps + 1))
+
+
+def paper_level_grid(G: int, group_size: int) -> Tuple[int, ...]:
+    """Remaining-structure counts of the database the paper builds per module (Sec. 3.2, "Runtime
+    awareness"; latency-table appendix): every head count G-1 .. 0 for an attention module; for an
+    FFN module the sizes of ``ffn_size_grid`` below G, repeated sizes dropped, and the dropped
+    module (0).  The unpruned size (i = 0) needs no pruning run and is left out."""
+    if group_size > 1:
+        return tuple(range(G - 1, -1, -1))
+    sizes = set(ffn_size_grid(G))
+    sizes.discard(G)
+    sizes.add(0)
+    return tuple(sorted(sizes, reverse=True))
+
+
 # The five workload families.  Names follow the model the shapes are taken from.
 CONFIGS = {
     # tiny single FFN-style layer, greedy to 75 % removed, snapshots at 25/50/75 %
