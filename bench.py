@@ -387,6 +387,44 @@ def run_ours(args, shape):
         del os.environ["ZIPLM_NEURON_PATH"]
     del os.environ["ZIPLM_LAYER_GROUPS"]
 
+    # ---- the Hessian from token-major activations (one token per row, the layout a forward pass
+    # emits): one call on the whole calibration set, and eight calibration batches with beta = 1
+    tok = None
+    if not args.skip_stream_leg:
+        A = X.transpose(1, 2).contiguous()
+        Ht = torch.empty_like(H)
+        t_ws = torch.empty(z.hessian_tokens_workspace_bytes(L, d, N, 0) + 256, dtype=torch.uint8,
+                           device=dev)
+        nb = 8
+        parts = [A[:, N * b // nb:N * (b + 1) // nb, :].contiguous() for b in range(nb)]
+
+        def whole():
+            z.hessian_accumulate_tokens(A, Ht, beta=0.0, workspace=t_ws)
+
+        def batched():
+            for b in range(nb):
+                z.hessian_accumulate_tokens(parts[b], Ht, beta=0.0 if b == 0 else 1.0, workspace=t_ws)
+
+        def plain():
+            z.hessian_accumulate(X, Ht, beta=0.0, workspace=h_ws)
+
+        tok = {}
+        for name, fn in (("feature_major_ms", plain), ("token_major_ms", whole),
+                         ("token_major_8_batches_ms", batched)):
+            for _ in range(2):
+                fn()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(5):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            tok[name] = e0.elapsed_time(e1) / 5
+        whole()
+        torch.cuda.synchronize()
+        tok["max_abs_diff_vs_feature_major"] = float((Ht - H).abs().max())
+        del A, parts, Ht, t_ws
+
     from paper_2302_04089_b200.parallel import max_over_ranks
     ms, ms_e2e = max_over_ranks(ms), max_over_ranks(ms_e2e)
     n_removed = G - min(levels)
@@ -468,6 +506,11 @@ def run_ours(args, shape):
                      "(ZIPLM_NEURON_PATH=stream), timed in a separate step",
                 phases_ms={k: round(v[0], 3) for k, v in phases_stream.items() if v[1] > 0}),
         )
+        if tok is not None:
+            tok["note"] = ("ziplm_hessian_accumulate_tokens on the same 12 x 3072 x 16384 fp32 "
+                           "activations stored one token per row; the transposing pre-pass replaces "
+                           "the split pre-pass (4 B read, 8 B written per element either way)")
+            line["hessian_token_major"] = tok
         if world == 1 and not args.no_cpu_baseline:
             s = oracle_sample(shape, n_loop_steps=args.oracle_steps)
             line["cpu_baseline"] = dict(

@@ -303,6 +303,67 @@ __global__ void __launch_bounds__(256) k_tokens_to_kmajor(const T* __restrict__ 
     }
 }
 
+// The same move for inputs whose rows allow 4-element vector accesses (A aligned to 4 elements,
+// lda % 4 == 0): a 64 x 64 tile, four elements per access on both sides, so a row of the output
+// leaves in 256-byte (fp32) pieces.  np is a multiple of 4, so a quad that starts below np ends
+// below it.
+template <typename T, typename V, bool SPLIT>
+__global__ void __launch_bounds__(256) k_tokens_to_kmajor_v4(const T* __restrict__ A, long long lda,
+                                                             long long N, int d, long long np,
+                                                             T* __restrict__ hi, T* __restrict__ lo) {
+    __shared__ T tile[64][65];                       // [token][feature]
+    union Quad { V v; T e[4]; };
+    const int l = blockIdx.z;
+    const long long t0 = (long long)blockIdx.x * 64;
+    const int f0 = blockIdx.y * 64;
+    const int q = threadIdx.x & 15, rr = threadIdx.x >> 4;
+    const T* Al = A + (size_t)l * (size_t)N * (size_t)lda;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int tl = rr + 16 * k;
+        const long long t = t0 + tl;
+        const int f = f0 + 4 * q;
+        Quad u;
+        if (t < N && f + 3 < d) {
+            u.v = *reinterpret_cast<const V*>(Al + (size_t)t * (size_t)lda + f);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                u.e[e] = (t < N && f + e < d) ? Al[(size_t)t * (size_t)lda + f + e] : T(0);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) tile[tl][4 * q + e] = u.e[e];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int fl = rr + 16 * k;
+        const int f = f0 + fl;
+        const long long t = t0 + 4 * q;
+        if (f >= d || t >= np) continue;
+        Quad u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) u.e[e] = tile[4 * q + e][fl];
+        const size_t o = ((size_t)l * d + f) * (size_t)np + (size_t)t;
+        if constexpr (SPLIT) {
+            Quad h, w;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                h.e[e] = __uint_as_float(__float_as_uint(u.e[e]) & 0xffffe000u);
+                w.e[e] = u.e[e] - h.e[e];
+            }
+            *reinterpret_cast<V*>(hi + o) = h.v;
+            *reinterpret_cast<V*>(lo + o) = w.v;
+        } else {
+            *reinterpret_cast<V*>(hi + o) = u.v;
+        }
+    }
+}
+
+bool quad_rows(const void* A, long long lda, size_t esz) {
+    return (reinterpret_cast<uintptr_t>(A) % (4 * esz)) == 0 && lda % 4 == 0;
+}
+
 // 3-D map over [layers, rows, K] with box {128 bytes of K, 128 rows, 1 layer}, 128-byte swizzle,
 // zero fill outside the tensor (ragged d and ragged token counts contribute zeros).
 bool make_map(CUtensorMap* m, const void* base, bool f32, long long K, int rows, int layers,
@@ -389,10 +450,16 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
                 // grid.z is limited to 65535 layers per launch
                 for (int z0 = 0; z0 < ln; z0 += 65535) {
                     const int zn = ln - z0 < 65535 ? ln - z0 : 65535;
-                    k_tokens_to_kmajor<float, true>
-                        <<<dim3((unsigned)((np + 31) / 32), (unsigned)((d + 31) / 32), (unsigned)zn), 256, 0,
-                           st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, np, hi + (size_t)z0 * d * np,
-                                 lo + (size_t)z0 * d * np);
+                    if (quad_rows(X, ldx, 4))
+                        k_tokens_to_kmajor_v4<float, float4, true>
+                            <<<dim3((unsigned)((np + 63) / 64), (unsigned)((d + 63) / 64), (unsigned)zn), 256,
+                               0, st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, np, hi + (size_t)z0 * d * np,
+                                        lo + (size_t)z0 * d * np);
+                    else
+                        k_tokens_to_kmajor<float, true>
+                            <<<dim3((unsigned)((np + 31) / 32), (unsigned)((d + 31) / 32), (unsigned)zn), 256,
+                               0, st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, np, hi + (size_t)z0 * d * np,
+                                        lo + (size_t)z0 * d * np);
                     ZIPLM_CHECK_LAUNCH();
                 }
             } else {
@@ -421,9 +488,14 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
         for (int l0 = 0; l0 < L; l0 += lc) {
             const int ln = (L - l0 < lc) ? (L - l0) : lc;
             const uint16_t* Ac = static_cast<const uint16_t*>(X) + (size_t)l0 * (size_t)N * ldx;
-            k_tokens_to_kmajor<uint16_t, false>
-                <<<dim3((unsigned)((np + 31) / 32), (unsigned)((d + 31) / 32), (unsigned)ln), 256, 0, st>>>(
-                    Ac, ldx, N, d, np, xt, nullptr);
+            if (quad_rows(X, ldx, 2))
+                k_tokens_to_kmajor_v4<uint16_t, uint2, false>
+                    <<<dim3((unsigned)((np + 63) / 64), (unsigned)((d + 63) / 64), (unsigned)ln), 256, 0, st>>>(
+                        Ac, ldx, N, d, np, xt, nullptr);
+            else
+                k_tokens_to_kmajor<uint16_t, false>
+                    <<<dim3((unsigned)((np + 31) / 32), (unsigned)((d + 31) / 32), (unsigned)ln), 256, 0, st>>>(
+                        Ac, ldx, N, d, np, xt, nullptr);
             ZIPLM_CHECK_LAUNCH();
             CUtensorMap mx;
             if (!make_map(&mx, xt, false, N, d, ln, np)) return ZIPLM_ERR_CUDA;

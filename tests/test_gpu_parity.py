@@ -86,7 +86,7 @@ def token_major_case(dtype, d, N, lda, L=2):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d,N,lda", [(64, 256, 64), (200, 1000, 208), (130, 613, 131), (96, 8, 96),
-                                     (33, 31, 40), (257, 4099, 257)])
+                                     (33, 31, 40), (257, 4099, 257), (130, 613, 132), (257, 4099, 260)])
 def test_hessian_from_token_major_activations_matches_oracle(dtype, d, N, lda):
     z = zb()
     X, A = token_major_case(dtype, d, N, lda)
