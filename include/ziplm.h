@@ -210,6 +210,49 @@ ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row
                                 size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Model reshaping (Sec. 3.1, "Pruned structures": once the columns of the removed structures are
+ * zero, the matching rows of the previous layer can be removed without any output change).
+ *
+ * A snapshot of ziplm_prune_layers keeps the original shape with zero columns.  These three calls
+ * turn a level of the database into the smaller dense matrices a runtime executes:
+ *
+ *   ziplm_kept_structures   kept[l] = the `level` structures of layer l that order[l][0 .. G-level)
+ *                           does not list, ascending
+ *   ziplm_gather_columns    out[l][i][k*g + c] = M[l][i][kept[l][k]*g + c]     (this layer: FC2,
+ *                           attention out-projection)
+ *   ziplm_gather_rows       out[l][k*g + c][j] = M[l][kept[l][k]*g + c][j]     (previous layer: FC1
+ *                           weight and, as a one-column matrix, its bias; the Q, K, V rows of a head)
+ *
+ * All three only move data; the outputs are bit-exact copies.
+ *
+ *   order         dev, [L, G] int, as written by ziplm_prune_layers; only the first G - level
+ *                 entries of a row are read
+ *   kept          dev, [L, level] int
+ *   layer_status  dev, [L] int: ZIPLM_OK, or ZIPLM_ERR_INVALID_ARG when those entries are not
+ *                 distinct indices in [0, G) (kept[l] is then unspecified)
+ *   M             dev, fp32; layer l starts at M + l * layer_stride (elements), row pitch ld
+ *                 (elements).  To read level slot s of W_snap [L, n_levels, d_row, d_col] pass
+ *                 W_snap + s * d_row * d_col, ld = d_col, layer_stride = n_levels * d_row * d_col.
+ *   rows / cols   number of rows of M (columns gather) / of columns of M that are copied (rows
+ *                 gather)
+ *   out           dev, dense [L, rows, level * g] (columns) or [L, level * g, cols] (rows)
+ *
+ * An entry of `kept` outside [0, G) produces zeros in the gathers.  level = 0 writes nothing.
+ * Errors: ZIPLM_ERR_INVALID_ARG (sizes, NULL pointers, ld smaller than the matrix width),
+ * ZIPLM_ERR_UNSUPPORTED (G beyond 1.6 million structures, rows beyond 1048560), ZIPLM_ERR_CUDA.
+ */
+ziplm_status ziplm_kept_structures(const int* order, int L, int G, int level, int* kept,
+                                   int* layer_status, void* cuda_stream);
+
+ziplm_status ziplm_gather_columns(const float* M, long long ld, long long layer_stride,
+                                  const int* kept, int L, int rows, int G, int group_size, int level,
+                                  float* out, void* cuda_stream);
+
+ziplm_status ziplm_gather_rows(const float* M, long long ld, long long layer_stride, const int* kept,
+                               int L, int cols, int G, int group_size, int level, float* out,
+                               void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Diagnostics (no counterpart in the paper): a launch counter and optional per-phase timing.
  *
  * ziplm_launch_count       kernels launched by this library since it was loaded.

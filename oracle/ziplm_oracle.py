@@ -260,3 +260,29 @@ def saliencies_on_support(W0, H_lam, remaining_groups: Sequence[int], group_size
         S = slice(k * g, (k + 1) * g)
         rho[k] = np.sum(Wc[:, S].T * np.linalg.solve(Hrr_inv[S, S], Wc[:, S].T))
     return groups, rho
+
+
+# --------------------------------------------------------------------------------------------
+# Model reshaping ("Pruned structures" paragraph of Sec. 3.1)
+# --------------------------------------------------------------------------------------------
+def kept_structures(order: Sequence[int], G: int, level: int) -> np.ndarray:
+    """The `level` structures that the first G - level removals leave, ascending."""
+    removed = [int(s) for s in order[:G - level]]
+    if len(set(removed)) != len(removed) or any(s < 0 or s >= G for s in removed):
+        raise ValueError("order must list distinct structures in [0, G)")
+    return np.array([s for s in range(G) if s not in set(removed)], dtype=np.int64)
+
+
+def drop_pruned_columns(W_masked, kept: Sequence[int], group_size: int) -> np.ndarray:
+    """This layer after reshaping: only the columns of the kept structures remain."""
+    W_masked = np.asarray(W_masked)
+    cols = [s * group_size + c for s in kept for c in range(group_size)]
+    return W_masked[:, cols]
+
+
+def drop_matching_rows(M_prev, kept: Sequence[int], group_size: int) -> np.ndarray:
+    """The previous layer after reshaping: the rows that produced the removed columns' inputs are
+    removed ("corresponding rows in previous layers can be safely removed")."""
+    M_prev = np.asarray(M_prev)
+    rows = [s * group_size + c for s in kept for c in range(group_size)]
+    return M_prev[rows]

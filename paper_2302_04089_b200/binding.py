@@ -78,6 +78,12 @@ def load_library() -> ctypes.CDLL:
     lib.ziplm_prune_layers.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_f,
                                        ctypes.POINTER(c_int), c_int, vp, vp, vp, vp, vp, vp, vp,
                                        c_sz, vp]
+    lib.ziplm_kept_structures.restype = c_int
+    lib.ziplm_kept_structures.argtypes = [vp, c_int, c_int, c_int, vp, vp, vp]
+    lib.ziplm_gather_columns.restype = c_int
+    lib.ziplm_gather_columns.argtypes = [vp, c_ll, c_ll, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
+    lib.ziplm_gather_rows.restype = c_int
+    lib.ziplm_gather_rows.argtypes = [vp, c_ll, c_ll, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
     lib.ziplm_launch_count.restype = ctypes.c_longlong
     lib.ziplm_launch_count.argtypes = []
     lib.ziplm_profile_begin.restype = c_int
@@ -273,6 +279,64 @@ def prune_layers(W: torch.Tensor, H: torch.Tensor, group_size: int, damp_frac: f
     if st != 0:
         raise ZiplmError(st, "ziplm_prune_layers")
     out["workspace"] = workspace
+    return out
+
+
+def kept_structures(order: torch.Tensor, level: int):
+    """(kept [L, level] int32 ascending, layer_status [L] int32) from the removal order [L, G] of
+    prune_layers; see ziplm_kept_structures."""
+    lib = load_library()
+    _check(order, torch.int32, "order")
+    L, G = order.shape
+    kept = torch.empty(L, max(level, 0), dtype=torch.int32, device=order.device)
+    status = torch.empty(L, dtype=torch.int32, device=order.device)
+    with torch.cuda.device(order.device):
+        st = lib.ziplm_kept_structures(order.data_ptr(), L, G, level, kept.data_ptr(),
+                                       status.data_ptr(), _stream_ptr(order))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_kept_structures")
+    return kept, status
+
+
+def _strided_layers(M: torch.Tensor, name: str):
+    if M.dim() != 3 or not M.is_cuda or M.dtype != torch.float32 or (M.shape[2] > 1 and M.stride(2) != 1):
+        raise ValueError(f"{name} must be a CUDA fp32 tensor [L, rows, cols] with contiguous rows")
+    return M.stride(1) if M.shape[1] > 1 else M.shape[2], M.stride(0) if M.shape[0] > 1 else 0
+
+
+def gather_columns(M: torch.Tensor, kept: torch.Tensor, group_size: int) -> torch.Tensor:
+    """out[l, i, k*g + c] = M[l, i, kept[l, k]*g + c]; M [L, rows, G*g] fp32 (may be a strided view,
+    e.g. ``W_snap[:, slot]``); see ziplm_gather_columns."""
+    lib = load_library()
+    ld, ls = _strided_layers(M, "M")
+    _check(kept, torch.int32, "kept")
+    L, rows, width = M.shape
+    level = kept.shape[1]
+    G = width // group_size
+    out = torch.empty(L, rows, level * group_size, dtype=torch.float32, device=M.device)
+    with torch.cuda.device(M.device):
+        st = lib.ziplm_gather_columns(M.data_ptr(), ld, ls, kept.data_ptr(), L, rows, G, group_size,
+                                      level, out.data_ptr(), _stream_ptr(M))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_gather_columns")
+    return out
+
+
+def gather_rows(M: torch.Tensor, kept: torch.Tensor, group_size: int) -> torch.Tensor:
+    """out[l, k*g + c, :] = M[l, kept[l, k]*g + c, :]; M [L, G*g, cols] fp32; see
+    ziplm_gather_rows."""
+    lib = load_library()
+    ld, ls = _strided_layers(M, "M")
+    _check(kept, torch.int32, "kept")
+    L, height, cols = M.shape
+    level = kept.shape[1]
+    G = height // group_size
+    out = torch.empty(L, level * group_size, cols, dtype=torch.float32, device=M.device)
+    with torch.cuda.device(M.device):
+        st = lib.ziplm_gather_rows(M.data_ptr(), ld, ls, kept.data_ptr(), L, cols, G, group_size,
+                                   level, out.data_ptr(), _stream_ptr(M))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_gather_rows")
     return out
 
 

@@ -146,4 +146,34 @@ ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row
                             workspace_bytes, st);
 }
 
+ziplm_status ziplm_kept_structures(const int* order, int L, int G, int level, int* kept,
+                                   int* layer_status, void* cuda_stream) {
+    if (L < 1 || G < 1 || level < 0 || level > G || !order || !layer_status) return ZIPLM_ERR_INVALID_ARG;
+    if (level > 0 && !kept) return ZIPLM_ERR_INVALID_ARG;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    return run_kept_structures(order, L, G, level, kept, layer_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
+ziplm_status ziplm_gather_columns(const float* M, long long ld, long long layer_stride, const int* kept,
+                                  int L, int rows, int G, int group_size, int level, float* out,
+                                  void* cuda_stream) {
+    if (L < 1 || rows < 0 || G < 1 || group_size < 1 || level < 0 || level > G) return ZIPLM_ERR_INVALID_ARG;
+    if (ld < (long long)G * group_size || layer_stride < 0) return ZIPLM_ERR_INVALID_ARG;
+    if (level > 0 && rows > 0 && (!M || !kept || !out)) return ZIPLM_ERR_INVALID_ARG;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    return run_gather_columns(M, ld, layer_stride, kept, L, rows, G, group_size, level, out,
+                              static_cast<cudaStream_t>(cuda_stream));
+}
+
+ziplm_status ziplm_gather_rows(const float* M, long long ld, long long layer_stride, const int* kept,
+                               int L, int cols, int G, int group_size, int level, float* out,
+                               void* cuda_stream) {
+    if (L < 1 || cols < 0 || G < 1 || group_size < 1 || level < 0 || level > G) return ZIPLM_ERR_INVALID_ARG;
+    if (ld < cols || layer_stride < 0) return ZIPLM_ERR_INVALID_ARG;
+    if (level > 0 && cols > 0 && (!M || !kept || !out)) return ZIPLM_ERR_INVALID_ARG;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    return run_gather_rows(M, ld, layer_stride, kept, L, cols, G, group_size, level, out,
+                           static_cast<cudaStream_t>(cuda_stream));
+}
+
 }  // extern "C"

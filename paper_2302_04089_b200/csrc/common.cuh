@@ -113,4 +113,12 @@ ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, bool token_maj
                          long long N, long long ldx, float alpha, float beta, void* ws,
                          size_t ws_bytes, cudaStream_t st);
 
+// Model reshaping (reshape.cu): survivors of a level, and column / row gathers by that list.
+ziplm_status run_kept_structures(const int* order, int L, int G, int level, int* kept, int* bad,
+                                 cudaStream_t st);
+ziplm_status run_gather_columns(const float* M, long long ld, long long layer_stride, const int* kept,
+                                int L, int rows, int G, int g, int level, float* out, cudaStream_t st);
+ziplm_status run_gather_rows(const float* M, long long ld, long long layer_stride, const int* kept,
+                             int L, int cols, int G, int g, int level, float* out, cudaStream_t st);
+
 }  // namespace ziplm

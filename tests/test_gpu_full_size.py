@@ -242,7 +242,25 @@ def test_paper_database_grid_from_streamed_token_major_batches():
     lockstep_head(Wl, H32, shape, out, l, 24)
     for slot in (0, 7, 21, 41, 42):          # sizes 2764, 1322, 302, 36, 0
         check_level(Wl, H32, shape, out, l, slot)
-    del W, out, H
+    # reshaping at full size: every layer's 302 survivors, columns of the snapshot (read in place)
+    # and rows of a stand-in FC1, bit for bit against plain indexing
+    lv, slot = 302, 21
+    kept, status = z.kept_structures(out["order"], lv)
+    fc1 = torch.randn(shape.n_layers, shape.d_col, 768, device="cuda",
+                      generator=torch.Generator(device="cuda").manual_seed(3))
+    Wc = z.gather_columns(out["W_snap"][:, slot], kept, 1)
+    Fc = z.gather_rows(fc1, kept, 1)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(status) == 0
+    order = out["order"].cpu().numpy()
+    for k in range(shape.n_layers):
+        ko = zo.kept_structures(order[k], shape.n_groups, lv)
+        assert np.array_equal(kept[k].cpu().numpy(), ko)
+        assert np.array_equal(Wc[k].cpu().numpy(),
+                              zo.drop_pruned_columns(out["W_snap"][k, slot].cpu().numpy(), ko, 1))
+        assert np.array_equal(Fc[k].cpu().numpy(), zo.drop_matching_rows(fc1[k].cpu().numpy(), ko, 1))
+        assert int(torch.count_nonzero(Wc[k])) == int(torch.count_nonzero(out["W_snap"][k, slot]))
+    del W, out, H, fc1, Wc, Fc
     torch.cuda.empty_cache()
 
     attn = wl.CONFIGS["c5_gpt2"][0]

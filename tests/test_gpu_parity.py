@@ -370,3 +370,63 @@ def test_invalid_arguments_are_rejected_on_the_host():
     with pytest.raises(z.ZiplmError) as e:
         z.prune_layers(W, H, 1, 0.01, [4], workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
     assert e.value.status == z.Status.ERR_WORKSPACE
+
+
+# ------------------------------------------------------------------ model reshaping
+@pytest.mark.parametrize("d,g,r,L,level", [(256, 1, 64, 2, 100), (384, 64, 96, 3, 2), (200, 4, 33, 2, 49),
+                                           (3072, 1, 40, 2, 302), (128, 1, 16, 1, 0), (128, 1, 16, 1, 128)])
+def test_reshaping_is_a_bit_exact_copy_of_the_kept_structures(d, g, r, L, level):
+    """Survivor list and both gathers against plain indexing, bit for bit, on the output of a real
+    pruning run (snapshot read in place through its strides) and on a stand-in previous layer."""
+    z = zb()
+    G = d // g
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2" if g == 1 else "c2_bert_base_attn"][0], d_row=r,
+                   d_col=d, d_latent=min(d, 96), n_tokens=max(2 * d, 512), n_layers=L, group_size=g)
+    W, X = wl.make_layers(sh, "cpu")
+    H = torch.stack([oracle_h32(X[l]) for l in range(L)])
+    levels = [lv for lv in (G - 1, level) if lv < G] or [level]
+    levels = sorted(set(levels), reverse=True)
+    out = z.prune_layers(W.cuda(), H.cuda(), g, sh.damp_frac, levels)
+    slot = levels.index(level) if level in levels else None
+    kept, status = z.kept_structures(out["order"], level)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(status) == 0
+    order = out["order"].cpu().numpy()
+    prev = torch.randn(L, d, 24, generator=torch.Generator().manual_seed(5))     # e.g. FC1 [d, d_in]
+    for l in range(L):
+        ko = zo.kept_structures(order[l], G, level)
+        assert np.array_equal(kept[l].cpu().numpy(), ko)
+    if level == G:
+        snap = W.cuda()                                     # nothing removed: the layer itself
+    else:
+        snap = out["W_snap"][:, slot]                       # strided view, read in place
+    Wc = z.gather_columns(snap, kept, g)
+    Pc = z.gather_rows(prev.cuda(), kept, g)
+    bias = z.gather_rows(prev.cuda()[:, :, :1].contiguous(), kept, g)
+    torch.cuda.synchronize()
+    assert Wc.shape == (L, r, level * g) and Pc.shape == (L, level * g, 24)
+    for l in range(L):
+        ko = kept[l].cpu().numpy()
+        assert np.array_equal(Wc[l].cpu().numpy(), zo.drop_pruned_columns(snap[l].cpu().numpy(), ko, g))
+        assert np.array_equal(Pc[l].cpu().numpy(), zo.drop_matching_rows(prev[l].numpy(), ko, g))
+        assert np.array_equal(bias[l].cpu().numpy(), zo.drop_matching_rows(prev[l][:, :1].numpy(), ko, g))
+        if level < G:
+            # the dropped columns were exactly zero: nothing of the snapshot is lost
+            assert int(torch.count_nonzero(Wc[l])) == int(torch.count_nonzero(snap[l]))
+
+
+def test_reshaping_rejects_a_level_the_order_does_not_reach():
+    z = zb()
+    order = torch.tensor([[3, 1, -1, -1], [2, 2, 0, 1]], dtype=torch.int32, device="cuda")
+    kept, status = z.kept_structures(order, 2)              # two removals: fine for layer 0 only
+    torch.cuda.synchronize()
+    assert status.tolist() == [0, int(z.Status.ERR_INVALID_ARG)]
+    assert kept[0].tolist() == [0, 2]
+    _, status = z.kept_structures(order, 1)                 # three removals: layer 0 ran only two
+    assert status.tolist() == [int(z.Status.ERR_INVALID_ARG)] * 2
+    with pytest.raises(z.ZiplmError):
+        z.kept_structures(order, 5)
+    # an index outside [0, G) in a caller-made list gives zeros, never an out-of-bounds read
+    M = torch.ones(1, 2, 4, device="cuda")
+    bad = torch.tensor([[1, 9]], dtype=torch.int32, device="cuda")
+    assert z.gather_columns(M, bad, 1).tolist() == [[[1.0, 0.0], [1.0, 0.0]]]

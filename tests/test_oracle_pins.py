@@ -455,3 +455,43 @@ def test_level_validation():
         zo.prune(W0, H, 1, 0.01, [9])
     with pytest.raises(ValueError):
         zo.GreedyOBS(W0, np.eye(8), 3)
+
+
+# ------------------------------------------------------------------ model reshaping
+@pytest.mark.parametrize("g", [1, 2])
+def test_reshaped_two_layer_block_computes_the_same_output(g):
+    """"Pruned structures" (Sec. 3.1): with the removed columns of the second matrix zero, dropping
+    them and the matching rows (and bias entries) of the first matrix changes no output -- checked
+    on a small FC1 -> GELU -> FC2 block against the masked, full-shape block."""
+    rng = np.random.default_rng(21)
+    d_in, d_mid, d_out, N = 5, 12, 4, 9
+    W1, b1 = rng.normal(size=(d_mid, d_in)), rng.normal(size=d_mid)
+    W2 = rng.normal(size=(d_out, d_mid))
+    inp = rng.normal(size=(d_in, N))
+    import math
+    erf = np.vectorize(math.erf)
+
+    def act(v):                                                       # exact GELU
+        return 0.5 * v * (1.0 + erf(v / np.sqrt(2.0)))
+
+    X = act(W1 @ inp + b1[:, None])                                   # inputs of the pruned layer
+    G = d_mid // g
+    res = zo.prune(W2, zo.hessian(X), g, 0.01, [G // 2])
+    W_masked = res["snapshots"][G // 2]
+    kept = zo.kept_structures(res["order"], G, G // 2)
+    assert len(kept) == G // 2 and list(kept) == sorted(set(range(G)) - set(res["order"][:G - G // 2]))
+    W2c = zo.drop_pruned_columns(W_masked, kept, g)
+    W1c = zo.drop_matching_rows(W1, kept, g)
+    b1c = zo.drop_matching_rows(b1[:, None], kept, g)[:, 0]
+    assert W2c.shape == (d_out, (G // 2) * g) and W1c.shape == ((G // 2) * g, d_in)
+    full = W_masked @ X
+    small = W2c @ act(W1c @ inp + b1c[:, None])
+    assert np.allclose(full, small, rtol=1e-12, atol=1e-13)
+    # a wrong index map (e.g. keeping the removed structures instead) does change the output
+    wrong = [s for s in range(G) if s not in set(kept)]
+    if len(wrong) == len(kept):
+        W2w = zo.drop_pruned_columns(W_masked, wrong, g)
+        assert not np.allclose(full, W2w @ act(zo.drop_matching_rows(W1, wrong, g) @ inp
+                                               + zo.drop_matching_rows(b1[:, None], wrong, g)))
+    with pytest.raises(ValueError):
+        zo.kept_structures([0, 0], G, G - 2)
