@@ -253,6 +253,47 @@ ziplm_status ziplm_gather_rows(const float* M, long long ld, long long layer_str
                                void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Budgeted choice of one database level per module (Sec. 3.2, "Runtime awareness", "Finding the
+ * optimal sparsity configuration", "Structured SPDY search").
+ *
+ * For module m (an attention block or a fully-connected block) the database holds n_options[m]
+ * levels; level s costs time[m][s] in the latency table and has the prior
+ *     p[m][s] = loss[m][s] / base_loss[m]          (relative layer-wise squared error; 1 for a
+ *                                                   dropped module, 0 for the unpruned one)
+ * taken directly from the outputs of ziplm_prune_layers.  For each of n_candidates sensitivity
+ * vectors c[k] the call finds the levels that minimise  sum_m c[k][m] * p[m][s_m]  subject to
+ * sum_m time[m][s_m] <= budget.  The search of the paper solves this once per mutated coefficient
+ * vector (1000 steps), which is why candidates are batched.
+ *
+ * Time is discretised into n_buckets units of budget / n_buckets and every option is rounded UP
+ * (units = ceil(time * n_buckets / budget) in float64), so the selection never exceeds the budget
+ * in real time; it is optimal for the discretised problem.  Costs are float64 sums formed in
+ * module order; ties go to the lowest option index.
+ *
+ *   loss, time        dev, [n_modules, max_options] fp32; entries s >= n_options[m] are ignored
+ *   base_loss         dev, [n_modules] fp32, > 0
+ *   n_options         dev, [n_modules] int, each in [1, max_options]
+ *   coef              dev, [n_candidates, n_modules] fp32
+ *   budget            total run time allowed, same unit as `time`, > 0
+ *   selected          dev, [n_candidates, n_modules] int: chosen option per module (-1 on failure)
+ *   cost              dev, [n_candidates] fp64: the minimum
+ *   time_sum          dev, [n_candidates] fp64: sum of the chosen options' times
+ *   candidate_status  dev, [n_candidates] int: ZIPLM_OK; ZIPLM_ERR_INVALID_ARG when even the
+ *                     fastest options exceed the budget; ZIPLM_ERR_NONFINITE for NaN inputs
+ *   workspace         dev scratch >= ziplm_select_workspace_bytes(...), 256-byte aligned
+ *
+ * Errors: ZIPLM_ERR_INVALID_ARG; ZIPLM_ERR_UNSUPPORTED (max_options > 255 or n_buckets > 12000);
+ * ZIPLM_ERR_WORKSPACE; ZIPLM_ERR_CUDA.
+ */
+size_t ziplm_select_workspace_bytes(int n_candidates, int n_modules, int n_buckets);
+
+ziplm_status ziplm_select_levels(const float* loss, const float* base_loss, const float* time,
+                                 const int* n_options, int n_modules, int max_options,
+                                 const float* coef, int n_candidates, double budget, int n_buckets,
+                                 int* selected, double* cost, double* time_sum, int* candidate_status,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Diagnostics (no counterpart in the paper): a launch counter and optional per-phase timing.
  *
  * ziplm_launch_count       kernels launched by this library since it was loaded.

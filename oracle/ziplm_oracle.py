@@ -286,3 +286,65 @@ def drop_matching_rows(M_prev, kept: Sequence[int], group_size: int) -> np.ndarr
     M_prev = np.asarray(M_prev)
     rows = [s * group_size + c for s in kept for c in range(group_size)]
     return M_prev[rows]
+
+
+# --------------------------------------------------------------------------------------------
+# Budgeted level selection (Sec. 3.2: "Runtime awareness", "Finding the optimal sparsity
+# configuration", "Structured SPDY search")
+# --------------------------------------------------------------------------------------------
+def error_prior(loss, base_loss) -> np.ndarray:
+    """p_s: the layer-wise squared error of level s relative to ||W X||^2 -- 1 for a dropped
+    module, 0 for the unpruned one ("Structured SPDY search")."""
+    return as_f64(loss) / as_f64(base_loss)
+
+
+def time_units(time, budget: float, n_buckets: int) -> int:
+    """Run time of one option in units of budget / n_buckets, rounded up so that a selection that
+    fits in units also fits in real time."""
+    import math
+    return int(math.ceil(float(np.float64(time) * (np.float64(n_buckets) / np.float64(budget)))))
+
+
+def select_levels(loss, base_loss, time, n_options: Sequence[int], coef, budget: float,
+                  n_buckets: int):
+    """One level per module minimising sum_m coef[m] * p[m][s_m] subject to
+    sum_m time[m][s_m] <= budget, by dynamic programming over modules on the discretised time
+    axis: f_{m+1}[b] = min_s f_m[b - units(m, s)] + coef[m] * p[m][s], ties to the lowest s.
+
+    loss, time: [n_modules, max_options]; base_loss, coef: [n_modules].
+    Returns (selected option per module, minimal cost, summed time), or (None, inf, 0.0) when even
+    the fastest options exceed the budget."""
+    loss, time, coef = as_f64(loss), as_f64(time), as_f64(coef)
+    base_loss = as_f64(base_loss)
+    n_mod = loss.shape[0]
+    f = np.zeros(n_buckets + 1)
+    choices, units = [], []
+    for m in range(n_mod):
+        best = np.full(n_buckets + 1, np.inf)
+        arg = np.zeros(n_buckets + 1, dtype=np.int64)
+        um = []
+        for s in range(int(n_options[m])):
+            cost = coef[m] * (loss[m, s] / base_loss[m])
+            u = time_units(time[m, s], budget, n_buckets)
+            um.append(u)
+            if u < 0 or u > n_buckets:
+                continue
+            cand = np.full(n_buckets + 1, np.inf)
+            cand[u:] = f[:n_buckets + 1 - u] + cost
+            better = cand < best                      # strict: the lowest s wins a tie
+            best[better] = cand[better]
+            arg[better] = s
+        f = best
+        choices.append(arg)
+        units.append(um)
+    if not np.isfinite(f[n_buckets]):
+        return None, float("inf"), 0.0
+    b = n_buckets
+    selected = [0] * n_mod
+    t_sum = 0.0
+    for m in range(n_mod - 1, -1, -1):
+        s = int(choices[m][b])
+        selected[m] = s
+        t_sum += time[m, s]
+        b -= units[m][s]
+    return selected, float(f[n_buckets]), float(t_sum)

@@ -84,6 +84,11 @@ def load_library() -> ctypes.CDLL:
     lib.ziplm_gather_columns.argtypes = [vp, c_ll, c_ll, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
     lib.ziplm_gather_rows.restype = c_int
     lib.ziplm_gather_rows.argtypes = [vp, c_ll, c_ll, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
+    lib.ziplm_select_workspace_bytes.restype = c_sz
+    lib.ziplm_select_workspace_bytes.argtypes = [c_int, c_int, c_int]
+    lib.ziplm_select_levels.restype = c_int
+    lib.ziplm_select_levels.argtypes = [vp, vp, vp, vp, c_int, c_int, vp, c_int, ctypes.c_double, c_int,
+                                        vp, vp, vp, vp, vp, c_sz, vp]
     lib.ziplm_launch_count.restype = ctypes.c_longlong
     lib.ziplm_launch_count.argtypes = []
     lib.ziplm_profile_begin.restype = c_int
@@ -337,6 +342,47 @@ def gather_rows(M: torch.Tensor, kept: torch.Tensor, group_size: int) -> torch.T
                                    level, out.data_ptr(), _stream_ptr(M))
     if st != 0:
         raise ZiplmError(st, "ziplm_gather_rows")
+    return out
+
+
+def select_workspace_bytes(n_candidates: int, n_modules: int, n_buckets: int) -> int:
+    return int(load_library().ziplm_select_workspace_bytes(n_candidates, n_modules, n_buckets))
+
+
+def select_levels(loss: torch.Tensor, base_loss: torch.Tensor, time: torch.Tensor,
+                  n_options: torch.Tensor, coef: torch.Tensor, budget: float, n_buckets: int,
+                  workspace: Optional[torch.Tensor] = None) -> dict:
+    """One database level per module under a run-time budget, for every row of ``coef``
+    [n_candidates, n_modules]; see ziplm_select_levels.  Returns CUDA tensors selected
+    [n_candidates, n_modules] int32, cost and time_sum [n_candidates] float64, status int32."""
+    lib = load_library()
+    _check(loss, torch.float32, "loss")
+    _check(time, torch.float32, "time")
+    _check(base_loss, torch.float32, "base_loss")
+    _check(n_options, torch.int32, "n_options")
+    _check(coef, torch.float32, "coef")
+    n_mod, max_opt = loss.shape
+    K = coef.shape[0]
+    if tuple(time.shape) != (n_mod, max_opt) or base_loss.numel() != n_mod or \
+            n_options.numel() != n_mod or coef.shape[1] != n_mod:
+        raise ValueError("shapes: loss/time [n_modules, max_options], base_loss/n_options [n_modules], "
+                         "coef [n_candidates, n_modules]")
+    dev = loss.device
+    out = dict(selected=torch.empty(K, n_mod, dtype=torch.int32, device=dev),
+               cost=torch.empty(K, dtype=torch.float64, device=dev),
+               time_sum=torch.empty(K, dtype=torch.float64, device=dev),
+               status=torch.empty(K, dtype=torch.int32, device=dev))
+    if workspace is None:
+        workspace = _workspace(select_workspace_bytes(K, n_mod, n_buckets), dev)
+    with torch.cuda.device(dev):
+        st = lib.ziplm_select_levels(loss.data_ptr(), base_loss.data_ptr(), time.data_ptr(),
+                                     n_options.data_ptr(), n_mod, max_opt, coef.data_ptr(), K,
+                                     float(budget), n_buckets, out["selected"].data_ptr(),
+                                     out["cost"].data_ptr(), out["time_sum"].data_ptr(),
+                                     out["status"].data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                     _stream_ptr(loss))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_select_levels")
     return out
 
 

@@ -176,4 +176,28 @@ ziplm_status ziplm_gather_rows(const float* M, long long ld, long long layer_str
                            static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t ziplm_select_workspace_bytes(int n_candidates, int n_modules, int n_buckets) {
+    if (n_candidates < 1 || n_modules < 1 || n_buckets < 1) return 0;
+    return select_workspace_bytes(n_candidates, n_modules, n_buckets);
+}
+
+ziplm_status ziplm_select_levels(const float* loss, const float* base_loss, const float* time,
+                                 const int* n_options, int n_modules, int max_options,
+                                 const float* coef, int n_candidates, double budget, int n_buckets,
+                                 int* selected, double* cost, double* time_sum, int* candidate_status,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (n_modules < 1 || max_options < 1 || n_candidates < 1 || n_buckets < 1) return ZIPLM_ERR_INVALID_ARG;
+    if (!(budget > 0.0) || !isfinite(budget)) return ZIPLM_ERR_INVALID_ARG;
+    if (!loss || !base_loss || !time || !n_options || !coef || !selected || !cost || !time_sum ||
+        !candidate_status)
+        return ZIPLM_ERR_INVALID_ARG;
+    if (max_options > 255 || n_buckets > 12000) return ZIPLM_ERR_UNSUPPORTED;
+    const size_t need = select_workspace_bytes(n_candidates, n_modules, n_buckets);
+    if (!workspace || !aligned(workspace, kAlign) || workspace_bytes < need) return ZIPLM_ERR_WORKSPACE;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    return run_select_levels(loss, base_loss, time, n_options, n_modules, max_options, coef, n_candidates,
+                             budget, n_buckets, selected, cost, time_sum, candidate_status, workspace,
+                             workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
 }  // extern "C"

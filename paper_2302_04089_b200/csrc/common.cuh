@@ -121,4 +121,12 @@ ziplm_status run_gather_columns(const float* M, long long ld, long long layer_st
 ziplm_status run_gather_rows(const float* M, long long ld, long long layer_stride, const int* kept,
                              int L, int cols, int G, int g, int level, float* out, cudaStream_t st);
 
+// Budgeted level selection (select.cu): one level per module under a run-time budget, K
+// coefficient vectors per launch.
+size_t select_workspace_bytes(int K, int n_mod, int n_buckets);
+ziplm_status run_select_levels(const float* loss, const float* base_loss, const float* time,
+                               const int* n_opt, int n_mod, int max_opt, const float* coef, int K,
+                               double budget, int n_buckets, int* selected, double* cost, double* time_sum,
+                               int* status, void* ws, size_t ws_bytes, cudaStream_t st);
+
 }  // namespace ziplm

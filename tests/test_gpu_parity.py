@@ -430,3 +430,119 @@ def test_reshaping_rejects_a_level_the_order_does_not_reach():
     M = torch.ones(1, 2, 4, device="cuda")
     bad = torch.tensor([[1, 9]], dtype=torch.int32, device="cuda")
     assert z.gather_columns(M, bad, 1).tolist() == [[[1.0, 0.0], [1.0, 0.0]]]
+
+
+# ------------------------------------------------------------------ budgeted level selection
+def synthetic_database(seed, n_mod, max_opt):
+    """Losses / run times shaped like a pruning database: option 0 unpruned (loss 0), the last one
+    the dropped module (loss = base, time 0); ragged option counts."""
+    g = torch.Generator().manual_seed(seed)
+    n_opt = torch.randint(2, max_opt + 1, (n_mod,), generator=g, dtype=torch.int32)
+    base = torch.rand(n_mod, generator=g) * 4 + 1
+    loss = torch.zeros(n_mod, max_opt)
+    time = torch.zeros(n_mod, max_opt)
+    for m in range(n_mod):
+        k = int(n_opt[m])
+        t = torch.sort(torch.rand(k, generator=g) * 7.5 + 0.5, descending=True).values
+        e = torch.sort(torch.rand(k, generator=g)).values
+        t[-1], e[0], e[-1] = 0.0, 0.0, 1.0
+        time[m, :k], loss[m, :k] = t, e * base[m]
+        time[m, k:], loss[m, k:] = -5.0, float("nan")          # padding must never be read
+    return loss, base, time, n_opt
+
+
+@pytest.mark.parametrize("n_mod,max_opt,n_buckets,K", [(5, 4, 97, 3), (24, 44, 1000, 6), (24, 44, 10000, 2),
+                                                      (1, 2, 1, 1), (7, 255, 12000, 1)])
+def test_level_selection_matches_oracle_bit_for_bit(n_mod, max_opt, n_buckets, K):
+    z = zb()
+    loss, base, time, n_opt = synthetic_database(11 + n_mod, n_mod, max_opt)
+    g = torch.Generator().manual_seed(99)
+    coef = torch.rand(K, n_mod, generator=g) * 3 + 0.05
+    t_all = float(sum(time[m, 0] for m in range(n_mod)))
+    for frac in (1.3, 0.5, 0.11):
+        budget = frac * t_all
+        out = z.select_levels(loss.cuda(), base.cuda(), time.cuda(), n_opt.cuda(), coef.cuda(), budget,
+                              n_buckets)
+        torch.cuda.synchronize()
+        for k in range(K):
+            sel, cost, t_sum = zo.select_levels(loss.numpy(), base.numpy(), time.numpy(), n_opt.numpy(),
+                                                coef[k].numpy(), budget, n_buckets)
+            assert int(out["status"][k]) == 0
+            assert out["selected"][k].tolist() == sel
+            assert float(out["cost"][k]) == cost                         # same float64 sums, same order
+            assert abs(float(out["time_sum"][k]) - t_sum) <= 1e-12 * max(t_sum, 1.0)
+            assert float(out["time_sum"][k]) <= budget * (1 + 1e-12)
+
+
+def test_level_selection_infeasible_budget_nan_and_bad_args():
+    z = zb()
+    loss, base, time, n_opt = synthetic_database(3, 4, 3)
+    time2 = time.clone()
+    for m in range(4):
+        time2[m, int(n_opt[m]) - 1] = 1.0                     # no free option any more
+    coef = torch.ones(2, 4)
+    out = z.select_levels(loss.cuda(), base.cuda(), time2.cuda(), n_opt.cuda(), coef.cuda(), 3.9, 40)
+    assert out["status"].tolist() == [int(z.Status.ERR_INVALID_ARG)] * 2
+    assert out["selected"].flatten().tolist() == [-1] * 8
+    assert zo.select_levels(loss.numpy(), base.numpy(), time2.numpy(), n_opt.numpy(), coef[0].numpy(),
+                            3.9, 40)[0] is None
+    out = z.select_levels(loss.cuda(), base.cuda(), time2.cuda(), n_opt.cuda(), coef.cuda(), 4.0, 40)
+    assert out["status"].tolist() == [0, 0]
+    bad = loss.clone()
+    bad[1, 0] = float("nan")
+    out = z.select_levels(bad.cuda(), base.cuda(), time.cuda(), n_opt.cuda(), coef.cuda(), 10.0, 40)
+    assert out["status"].tolist() == [int(z.Status.ERR_NONFINITE)] * 2
+    with pytest.raises(z.ZiplmError) as e:
+        z.select_levels(loss.cuda(), base.cuda(), time.cuda(), n_opt.cuda(), coef.cuda(), 10.0, 12001)
+    assert e.value.status == z.Status.ERR_UNSUPPORTED
+    with pytest.raises(z.ZiplmError) as e:
+        z.select_levels(loss.cuda(), base.cuda(), time.cuda(), n_opt.cuda(), coef.cuda(), 0.0, 40)
+    assert e.value.status == z.Status.ERR_INVALID_ARG
+
+
+def test_database_to_selection_end_to_end():
+    """Prune two small modules (heads and neurons) on every level of the paper's grid, feed the
+    library's own losses to the selection, and compare the chosen levels with the oracle's on the
+    same numbers; then reshape the chosen levels."""
+    z = zb()
+    attn = wl.scaled(wl.CONFIGS["c2_bert_base_attn"][0], n_layers=2, d_row=64, d_col=256, n_tokens=1024,
+                     levels=wl.paper_level_grid(4, 64))
+    ffn = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], n_layers=2, d_row=64, d_col=256, d_latent=64,
+                    n_tokens=1024, levels=wl.paper_level_grid(256, 1))
+    rows_loss, rows_time, rows_base, n_opt, outs = [], [], [], [], []
+    max_opt = 1 + max(len(attn.levels), len(ffn.levels))
+    for sh, full_ms, ovh in ((attn, 7.9, 0.6), (ffn, 11.9, 0.6)):
+        W, X = wl.make_layers(sh, "cuda")
+        out = z.prune_layers(W, z.hessian_accumulate(X), sh.group_size, sh.damp_frac, list(sh.levels))
+        sizes = (sh.n_groups,) + tuple(sh.levels)                     # option 0 = unpruned
+        t = wl.make_latency_table(sizes, full_ms, ovh)
+        for l in range(sh.n_layers):
+            lo = torch.full((max_opt,), float("nan"))
+            lo[0] = 0.0
+            lo[1:len(sizes)] = out["loss"][l].cpu()
+            ti = torch.full((max_opt,), -1.0)
+            ti[:len(sizes)] = t
+            rows_loss.append(lo); rows_time.append(ti); n_opt.append(len(sizes))
+            rows_base.append(out["base_loss"][l].cpu())
+        outs.append((sh, out))
+    loss, time = torch.stack(rows_loss), torch.stack(rows_time)
+    base, n_opt = torch.stack(rows_base), torch.tensor(n_opt, dtype=torch.int32)
+    coef = torch.ones(1, 4)
+    budget = 0.5 * float(time[:, 0].sum())                             # a 2x speedup target
+    res = z.select_levels(loss.cuda(), base.cuda(), time.cuda(), n_opt.cuda(), coef.cuda(), budget, 10000)
+    sel, cost, t_sum = zo.select_levels(loss.numpy(), base.numpy(), time.numpy(), n_opt.numpy(),
+                                        coef[0].numpy(), budget, 10000)
+    assert res["status"].tolist() == [0] and res["selected"][0].tolist() == sel
+    assert float(res["cost"][0]) == cost and float(res["time_sum"][0]) <= budget
+    assert 0.0 < cost < 4.0 and any(s > 0 for s in sel)
+    # reshape the FFN modules at their chosen levels
+    sh, out = outs[1]
+    for l in range(2):
+        s = sel[2 + l]
+        if s == 0:
+            continue
+        lv = sh.levels[s - 1]
+        kept, status = z.kept_structures(out["order"][l:l + 1].contiguous(), lv)
+        Wc = z.gather_columns(out["W_snap"][l:l + 1, s - 1], kept, 1)
+        assert int(status[0]) == 0 and Wc.shape == (1, sh.d_row, lv)
+        assert int(torch.count_nonzero(Wc)) == int(torch.count_nonzero(out["W_snap"][l, s - 1]))

@@ -495,3 +495,73 @@ def test_reshaped_two_layer_block_computes_the_same_output(g):
                                                + zo.drop_matching_rows(b1[:, None], wrong, g)))
     with pytest.raises(ValueError):
         zo.kept_structures([0, 0], G, G - 2)
+
+
+# ------------------------------------------------------------------ budgeted level selection
+def random_database(rng, n_mod, max_opt):
+    """Per module: decreasing run times, increasing losses (level 0 of the list = unpruned:
+    loss 0; last = dropped: loss = base, time 0), as a pruning database looks."""
+    n_opt = rng.integers(2, max_opt + 1, size=n_mod)
+    loss = np.zeros((n_mod, max_opt), np.float32)
+    time = np.zeros((n_mod, max_opt), np.float32)
+    base = rng.uniform(1.0, 5.0, size=n_mod).astype(np.float32)
+    for m in range(n_mod):
+        k = n_opt[m]
+        t = np.sort(rng.uniform(0.5, 8.0, size=k))[::-1].copy()
+        t[-1] = 0.0
+        e = np.sort(rng.uniform(0.0, 1.0, size=k))
+        e[0], e[-1] = 0.0, 1.0
+        time[m, :k] = t
+        loss[m, :k] = e * base[m]
+    return loss, base, time, n_opt
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_level_selection_against_exhaustive_search(seed):
+    """Every combination of levels is enumerated: the dynamic programme must return a selection
+    that fits the budget in units and attains the smallest cost among all that do; it must also
+    fit in real time (options are rounded up)."""
+    import itertools
+    rng = np.random.default_rng(seed)
+    n_mod, max_opt, n_buckets = 5, 4, 97
+    loss, base, time, n_opt = random_database(rng, n_mod, max_opt)
+    coef = rng.uniform(0.1, 3.0, size=n_mod).astype(np.float32)
+    t_all = float(time[:, 0].sum())
+    for frac in (1.2, 0.7, 0.45, 0.2, 0.02):
+        budget = frac * t_all
+        sel, cost, t_sum = zo.select_levels(loss, base, time, n_opt, coef, budget, n_buckets)
+        best = np.inf
+        for combo in itertools.product(*[range(k) for k in n_opt]):
+            u = sum(zo.time_units(time[m, s], budget, n_buckets) for m, s in enumerate(combo))
+            if u <= n_buckets:
+                c = sum(float(coef[m]) * float(loss[m, s]) / float(base[m]) for m, s in enumerate(combo))
+                best = min(best, c)
+        assert sel is not None and np.isclose(cost, best, rtol=1e-12, atol=1e-15)
+        assert t_sum <= budget * (1 + 1e-12)
+        assert np.isclose(cost, sum(float(coef[m]) * float(loss[m, s]) / float(base[m])
+                                    for m, s in enumerate(sel)), rtol=1e-12, atol=1e-15)
+        if frac == 1.2:     # the unpruned model fits (even with every option rounded up): nothing is lost
+            assert sel == [0] * n_mod and cost == 0.0
+
+
+def test_level_selection_limits_and_monotonicity():
+    rng = np.random.default_rng(7)
+    loss, base, time, n_opt = random_database(rng, 6, 5)
+    coef = np.ones(6, np.float32)
+    # budget (almost) zero: only the dropped modules (time 0) fit; cost = sum of priors of 1
+    sel, cost, t_sum = zo.select_levels(loss, base, time, n_opt, coef, 1e-3, 50)
+    assert sel == [int(k) - 1 for k in n_opt] and np.isclose(cost, 6.0) and t_sum == 0.0
+    assert np.allclose(zo.error_prior(loss[np.arange(6), n_opt - 1], base), 1.0)
+    # more budget never costs more
+    costs = [zo.select_levels(loss, base, time, n_opt, coef, b, 200)[1] for b in (2.0, 5.0, 9.0, 20.0, 60.0)]
+    assert all(a >= b - 1e-12 for a, b in zip(costs, costs[1:]))
+    # a module nobody cares about (coefficient 0) is dropped first when time is short
+    coef2 = coef.copy()
+    coef2[2] = 0.0
+    sel2, _, _ = zo.select_levels(loss, base, time, n_opt, coef2, 0.5 * float(time[:, 0].sum()), 200)
+    assert sel2[2] == n_opt[2] - 1
+    # no option without run time 0 and a budget below the fastest configuration: infeasible
+    time3 = time.copy()
+    time3[np.arange(6), n_opt - 1] = 1.0
+    assert zo.select_levels(loss, base, time3, n_opt, coef, 5.9, 60)[0] is None
+    assert zo.select_levels(loss, base, time3, n_opt, coef, 6.0, 60)[0] == [int(k) - 1 for k in n_opt]

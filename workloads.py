@@ -153,3 +153,13 @@ def make_layers(shape: LayerShape, device: str = "cpu",
     W = torch.stack([make_weight(shape, l) for l in idx]).to(device)
     X = torch.stack([make_activations(shape, l, device) for l in idx])
     return W, X
+
+
+def make_latency_table(sizes: Tuple[int, ...], full_ms: float, overhead_ms: float) -> torch.Tensor:
+    """Synthetic stand-in for one column of the paper's latency table (latency-table appendix):
+    run time of a module against its remaining structures, affine in the size with a fixed
+    overhead, 0 for the dropped module.  The paper measures these on the target device; only the
+    shape of the table (monotone, overhead-dominated at small sizes) is kept."""
+    top = float(max(sizes))
+    return torch.tensor([0.0 if n == 0 else overhead_ms + (full_ms - overhead_ms) * n / top
+                         for n in sizes], dtype=torch.float32)
