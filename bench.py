@@ -455,6 +455,67 @@ def run_ours(args, shape):
                             "database; output buffers allocated by torch inside the timed region")
         del prev
 
+    # ---- budgeted level selection on a database of the paper's size: 24 modules (12 attention,
+    # 12 FFN), the paper's level grid, 10^4 time buckets; 1024 coefficient vectors per launch, and
+    # the 1000-step mutation search for 148 speedup targets at once (one CTA each)
+    select = None
+    if not args.skip_stream_leg:
+        gsel = torch.Generator().manual_seed(1)
+        grids = [wl.paper_level_grid(12, 64), wl.paper_level_grid(G, 1)]
+        max_opt = 1 + max(len(x) for x in grids)
+        n_mod = 24
+        s_loss = torch.zeros(n_mod, max_opt)
+        s_time = torch.full((n_mod, max_opt), -1.0)
+        s_nopt = torch.zeros(n_mod, dtype=torch.int32)
+        for m in range(n_mod):
+            sizes = ((12,) if m % 2 == 0 else (G,)) + grids[m % 2]
+            k = len(sizes)
+            s_nopt[m] = k
+            s_time[m, :k] = wl.make_latency_table(sizes, 7.9 if m % 2 == 0 else 11.9, 0.6)
+            # priors rise as the module shrinks: the bench layer's own loss curve where it has one
+            frac = torch.tensor([1.0 - n / sizes[0] for n in sizes])
+            s_loss[m, :k] = frac ** 2 * (0.5 + torch.rand(1, generator=gsel))
+        s_base = torch.ones(n_mod)
+        Ksel, S, n_steps, n_buckets = 1024, 148, 1000, 10000
+        coefs = (torch.rand(Ksel, n_mod, generator=gsel) * 3 + 0.05).to(dev)
+        dl, db, dt_, dn = s_loss.to(dev), s_base.to(dev), s_time.to(dev), s_nopt.to(dev)
+        budget = 0.5 * float(s_time[:, 0].sum())
+        ws_sel = torch.empty(z.select_workspace_bytes(Ksel, n_mod, n_buckets) + 256, dtype=torch.uint8,
+                             device=dev)
+        z.select_levels(dl, db, dt_, dn, coefs, budget, n_buckets, workspace=ws_sel)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(3):
+            res = z.select_levels(dl, db, dt_, dn, coefs, budget, n_buckets, workspace=ws_sel)
+        e1.record()
+        torch.cuda.synchronize()
+        sel_ms = e0.elapsed_time(e1) / 3
+        assert int(torch.count_nonzero(res["status"])) == 0
+        del ws_sel
+        mask = (torch.rand(S, n_steps, n_mod, generator=gsel) < 0.1).to(torch.uint8).to(dev)
+        vals = (torch.rand(S, n_steps, n_mod, generator=gsel) * 3 + 0.05).to(dev)
+        budgets = (torch.linspace(0.08, 0.9, S, dtype=torch.float64) * float(s_time[:, 0].sum())).to(dev)
+        obj = (dl * (torch.rand(n_mod, 1, generator=gsel) + 0.5).to(dev)).contiguous()
+        coef0 = torch.ones(S, n_mod, device=dev)
+        e0.record()
+        sres = z.search_levels(dl, db, dt_, dn, obj, coef0, budgets, n_buckets, mask, vals)
+        e1.record()
+        torch.cuda.synchronize()
+        search_ms = e0.elapsed_time(e1)
+        assert int(torch.count_nonzero(sres["status"])) == 0
+        inner = float(sum(int(k) for k in s_nopt)) * (n_buckets + 1)
+        select = dict(modules=n_mod, max_options=max_opt, n_buckets=n_buckets,
+                      select_candidates=Ksel, select_ms=sel_ms,
+                      selections_per_sec=Ksel / (sel_ms * 1e-3),
+                      select_option_evals_per_sec=Ksel * inner / (sel_ms * 1e-3),
+                      search_targets=S, search_steps=n_steps, search_ms=search_ms,
+                      search_option_evals_per_sec=S * (n_steps + 1) * inner / (search_ms * 1e-3),
+                      mean_accepted=float(sres["n_accepted"].float().mean()),
+                      note="ziplm_select_levels / ziplm_search_levels on a synthetic database of the "
+                           "paper's size (latency table: affine stand-in); an option evaluation is one "
+                           "float64 add + compare against a shared-memory value row")
+        del mask, vals
+
     from paper_2302_04089_b200.parallel import max_over_ranks
     ms, ms_e2e = max_over_ranks(ms), max_over_ranks(ms_e2e)
     n_removed = G - min(levels)
@@ -543,6 +604,8 @@ def run_ours(args, shape):
             line["hessian_token_major"] = tok
         if reshape is not None:
             line["reshape_database"] = reshape
+        if select is not None:
+            line["level_selection"] = select
         if world == 1 and not args.no_cpu_baseline:
             s = oracle_sample(shape, n_loop_steps=args.oracle_steps)
             line["cpu_baseline"] = dict(

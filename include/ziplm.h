@@ -294,6 +294,51 @@ ziplm_status ziplm_select_levels(const float* loss, const float* base_loss, cons
                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Mutation search over the sensitivity coefficients (Sec. 3.2, "Structured SPDY search": a fixed
+ * number of steps -- 1000 in the paper -- each mutating in expectation 10 % of the coefficients).
+ *
+ * For each of n_searches run-time budgets (speedup targets), starting from coef0[k]: step t
+ * replaces the coefficients m with mask[k][t][m] != 0 by values[k][t][m], solves the selection
+ * problem of ziplm_select_levels for the mutated vector, scores the selection, and keeps the
+ * mutated vector when its score is strictly lower than the best so far (the unmutated coef0 is
+ * scored first).  The random draws are the caller's: marks drawn with probability 0.1 per
+ * coefficient give the paper's mutation rate.
+ *
+ * Score: the paper scores a candidate by the calibration loss of the stitched model, which only
+ * the caller's model can give.  Here the score of a selection is sum_m objective[m][s_m], a
+ * separable stand-in (for instance priors measured against a held-out calibration set); a caller
+ * with a model uses ziplm_select_levels on a batch of mutated vectors and scores them itself.
+ * Every selection the search evaluates meets its budget, as in the paper.
+ *
+ *   loss, base_loss, time, n_options, n_modules, max_options, n_buckets
+ *                    as for ziplm_select_levels
+ *   objective        dev, [n_modules, max_options] fp32
+ *   coef0            dev, [n_searches, n_modules] fp32
+ *   budgets          dev, [n_searches] fp64, each > 0
+ *   mask             dev, [n_searches, n_steps, n_modules] bytes
+ *   values           dev, [n_searches, n_steps, n_modules] fp32
+ *   best_selected    dev, [n_searches, n_modules] int (-1 if no evaluated selection met the budget)
+ *   best_coef        dev, [n_searches, n_modules] fp32: the coefficients that produced it
+ *   best_objective   dev, [n_searches] fp64 (float64 sum in module order; inf if none)
+ *   n_accepted       dev, [n_searches] int: mutations that were kept
+ *   search_status    dev, [n_searches] int: ZIPLM_OK, ZIPLM_ERR_INVALID_ARG (budget below the
+ *                    fastest configuration), ZIPLM_ERR_NONFINITE
+ *   workspace        dev scratch >= ziplm_search_workspace_bytes(...), 256-byte aligned
+ *
+ * One thread block runs one whole search, so the call is efficient when many targets are searched
+ * together.  Errors: as ziplm_select_levels; ZIPLM_ERR_UNSUPPORTED also for n_modules > 512.
+ */
+size_t ziplm_search_workspace_bytes(int n_searches, int n_modules, int n_buckets);
+
+ziplm_status ziplm_search_levels(const float* loss, const float* base_loss, const float* time,
+                                 const int* n_options, int n_modules, int max_options,
+                                 const float* objective, const float* coef0, const double* budgets,
+                                 int n_searches, int n_buckets, const unsigned char* mask,
+                                 const float* values, int n_steps, int* best_selected, float* best_coef,
+                                 double* best_objective, int* n_accepted, int* search_status,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Diagnostics (no counterpart in the paper): a launch counter and optional per-phase timing.
  *
  * ziplm_launch_count       kernels launched by this library since it was loaded.

@@ -348,3 +348,31 @@ def select_levels(loss, base_loss, time, n_options: Sequence[int], coef, budget:
         t_sum += time[m, s]
         b -= units[m][s]
     return selected, float(f[n_buckets]), float(t_sum)
+
+
+def search_levels(loss, base_loss, time, n_options, objective, coef0, budget: float, n_buckets: int,
+                  mask, values):
+    """The mutation search of "Structured SPDY search", step by step: score coef0; then for every
+    step replace the marked coefficients by the given values, solve the selection problem, score
+    the selection (sum over modules of objective[m][s_m], the stand-in for the stitched model's
+    calibration loss) and keep the mutated vector if the score is strictly lower.  mask, values:
+    [n_steps, n_modules], drawn by the caller.
+    Returns (best selection or None, best coefficients, best score, number of accepted steps)."""
+    objective = as_f64(objective)
+    best_c = np.asarray(coef0, dtype=np.float32).copy()
+    best_sel, best_score, accepted = None, float("inf"), 0
+    for step in range(len(mask) + 1):
+        c = best_c.copy()
+        if step > 0:
+            marked = np.asarray(mask[step - 1]) != 0
+            c[marked] = np.asarray(values[step - 1], dtype=np.float32)[marked]
+        sel, _, _ = select_levels(loss, base_loss, time, n_options, c, budget, n_buckets)
+        if sel is None:
+            continue
+        score = 0.0
+        for m, s in enumerate(sel):
+            score += objective[m, s]
+        if score < best_score:
+            best_sel, best_score, best_c = sel, score, c
+            accepted += step > 0
+    return best_sel, best_c, best_score, int(accepted)

@@ -89,6 +89,11 @@ def load_library() -> ctypes.CDLL:
     lib.ziplm_select_levels.restype = c_int
     lib.ziplm_select_levels.argtypes = [vp, vp, vp, vp, c_int, c_int, vp, c_int, ctypes.c_double, c_int,
                                         vp, vp, vp, vp, vp, c_sz, vp]
+    lib.ziplm_search_workspace_bytes.restype = c_sz
+    lib.ziplm_search_workspace_bytes.argtypes = [c_int, c_int, c_int]
+    lib.ziplm_search_levels.restype = c_int
+    lib.ziplm_search_levels.argtypes = [vp, vp, vp, vp, c_int, c_int, vp, vp, vp, c_int, c_int, vp, vp,
+                                        c_int, vp, vp, vp, vp, vp, vp, c_sz, vp]
     lib.ziplm_launch_count.restype = ctypes.c_longlong
     lib.ziplm_launch_count.argtypes = []
     lib.ziplm_profile_begin.restype = c_int
@@ -383,6 +388,51 @@ def select_levels(loss: torch.Tensor, base_loss: torch.Tensor, time: torch.Tenso
                                      _stream_ptr(loss))
     if st != 0:
         raise ZiplmError(st, "ziplm_select_levels")
+    return out
+
+
+def search_workspace_bytes(n_searches: int, n_modules: int, n_buckets: int) -> int:
+    return int(load_library().ziplm_search_workspace_bytes(n_searches, n_modules, n_buckets))
+
+
+def search_levels(loss: torch.Tensor, base_loss: torch.Tensor, time: torch.Tensor,
+                  n_options: torch.Tensor, objective: torch.Tensor, coef0: torch.Tensor,
+                  budgets: torch.Tensor, n_buckets: int, mask: torch.Tensor, values: torch.Tensor,
+                  workspace: Optional[torch.Tensor] = None) -> dict:
+    """Mutation search over the sensitivity coefficients, one search per budget; see
+    ziplm_search_levels.  mask [S, n_steps, n_modules] uint8, values the same shape fp32."""
+    lib = load_library()
+    for t, dt, name in ((loss, torch.float32, "loss"), (time, torch.float32, "time"),
+                        (base_loss, torch.float32, "base_loss"), (n_options, torch.int32, "n_options"),
+                        (objective, torch.float32, "objective"), (coef0, torch.float32, "coef0"),
+                        (budgets, torch.float64, "budgets"), (mask, torch.uint8, "mask"),
+                        (values, torch.float32, "values")):
+        _check(t, dt, name)
+    n_mod, max_opt = loss.shape
+    S, n_steps = mask.shape[0], mask.shape[1]
+    if tuple(mask.shape) != (S, n_steps, n_mod) or tuple(values.shape) != (S, n_steps, n_mod) or \
+            tuple(coef0.shape) != (S, n_mod) or budgets.numel() != S or \
+            tuple(objective.shape) != (n_mod, max_opt) or tuple(time.shape) != (n_mod, max_opt):
+        raise ValueError("shapes: mask/values [S, n_steps, n_modules], coef0 [S, n_modules], budgets [S]")
+    dev = loss.device
+    out = dict(selected=torch.empty(S, n_mod, dtype=torch.int32, device=dev),
+               coef=torch.empty(S, n_mod, dtype=torch.float32, device=dev),
+               objective=torch.empty(S, dtype=torch.float64, device=dev),
+               n_accepted=torch.empty(S, dtype=torch.int32, device=dev),
+               status=torch.empty(S, dtype=torch.int32, device=dev))
+    if workspace is None:
+        workspace = _workspace(search_workspace_bytes(S, n_mod, n_buckets), dev)
+    with torch.cuda.device(dev):
+        st = lib.ziplm_search_levels(loss.data_ptr(), base_loss.data_ptr(), time.data_ptr(),
+                                     n_options.data_ptr(), n_mod, max_opt, objective.data_ptr(),
+                                     coef0.data_ptr(), budgets.data_ptr(), S, n_buckets,
+                                     mask.data_ptr(), values.data_ptr(), n_steps,
+                                     out["selected"].data_ptr(), out["coef"].data_ptr(),
+                                     out["objective"].data_ptr(), out["n_accepted"].data_ptr(),
+                                     out["status"].data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                     _stream_ptr(loss))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_search_levels")
     return out
 
 

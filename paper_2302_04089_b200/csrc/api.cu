@@ -200,4 +200,32 @@ ziplm_status ziplm_select_levels(const float* loss, const float* base_loss, cons
                              workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t ziplm_search_workspace_bytes(int n_searches, int n_modules, int n_buckets) {
+    if (n_searches < 1 || n_modules < 1 || n_buckets < 1) return 0;
+    return search_workspace_bytes(n_searches, n_modules, n_buckets);
+}
+
+ziplm_status ziplm_search_levels(const float* loss, const float* base_loss, const float* time,
+                                 const int* n_options, int n_modules, int max_options,
+                                 const float* objective, const float* coef0, const double* budgets,
+                                 int n_searches, int n_buckets, const unsigned char* mask,
+                                 const float* values, int n_steps, int* best_selected, float* best_coef,
+                                 double* best_objective, int* n_accepted, int* search_status,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (n_modules < 1 || max_options < 1 || n_searches < 1 || n_buckets < 1 || n_steps < 0)
+        return ZIPLM_ERR_INVALID_ARG;
+    if (!loss || !base_loss || !time || !n_options || !objective || !coef0 || !budgets || !best_selected ||
+        !best_coef || !best_objective || !n_accepted || !search_status)
+        return ZIPLM_ERR_INVALID_ARG;
+    if (n_steps > 0 && (!mask || !values)) return ZIPLM_ERR_INVALID_ARG;
+    if (max_options > 255 || n_buckets > 12000 || n_modules > 512) return ZIPLM_ERR_UNSUPPORTED;
+    const size_t need = search_workspace_bytes(n_searches, n_modules, n_buckets);
+    if (!workspace || !aligned(workspace, kAlign) || workspace_bytes < need) return ZIPLM_ERR_WORKSPACE;
+    if (!have_device()) return ZIPLM_ERR_CUDA;
+    return run_search_levels(loss, base_loss, time, n_options, n_modules, max_options, objective, coef0,
+                             budgets, n_searches, n_buckets, mask, values, n_steps, best_selected, best_coef,
+                             best_objective, n_accepted, search_status, workspace, workspace_bytes,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
 }  // extern "C"

@@ -129,4 +129,12 @@ ziplm_status run_select_levels(const float* loss, const float* base_loss, const 
                                double budget, int n_buckets, int* selected, double* cost, double* time_sum,
                                int* status, void* ws, size_t ws_bytes, cudaStream_t st);
 
+size_t search_workspace_bytes(int S, int n_mod, int n_buckets);
+ziplm_status run_search_levels(const float* loss, const float* base_loss, const float* time,
+                               const int* n_opt, int n_mod, int max_opt, const float* objective,
+                               const float* coef0, const double* budgets, int S, int n_buckets,
+                               const unsigned char* mask, const float* values, int n_steps, int* best_sel,
+                               float* best_coef, double* best_obj, int* n_accepted, int* status, void* ws,
+                               size_t ws_bytes, cudaStream_t st);
+
 }  // namespace ziplm

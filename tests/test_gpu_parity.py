@@ -546,3 +546,40 @@ def test_database_to_selection_end_to_end():
         Wc = z.gather_columns(out["W_snap"][l:l + 1, s - 1], kept, 1)
         assert int(status[0]) == 0 and Wc.shape == (1, sh.d_row, lv)
         assert int(torch.count_nonzero(Wc)) == int(torch.count_nonzero(out["W_snap"][l, s - 1]))
+
+
+@pytest.mark.parametrize("n_mod,max_opt,n_buckets,steps", [(24, 44, 1000, 40), (5, 4, 97, 25)])
+def test_mutation_search_matches_oracle_bit_for_bit(n_mod, max_opt, n_buckets, steps):
+    """Three speedup targets searched in one launch against the oracle's step-by-step loop on
+    the same marks and values: same accepted steps, same coefficients, same selection, same
+    float64 score."""
+    z = zb()
+    loss, base, time, n_opt = synthetic_database(40 + n_mod, n_mod, max_opt)
+    g = torch.Generator().manual_seed(7)
+    S = 3
+    coef0 = torch.ones(S, n_mod)
+    mask = (torch.rand(S, steps, n_mod, generator=g) < 0.1).to(torch.uint8)     # 10 % in expectation
+    values = torch.rand(S, steps, n_mod, generator=g) * 3 + 0.05
+    objective = torch.nan_to_num(loss / base[:, None] * (torch.rand(n_mod, 1, generator=g) + 0.5), nan=0.0)
+    t_all = float(sum(time[m, 0] for m in range(n_mod)))
+    budgets = torch.tensor([0.8 * t_all, 0.5 * t_all, 0.1 * t_all], dtype=torch.float64)
+    out = z.search_levels(loss.cuda(), base.cuda(), time.cuda(), n_opt.cuda(), objective.cuda(),
+                          coef0.cuda(), budgets.cuda(), n_buckets, mask.cuda(), values.cuda())
+    torch.cuda.synchronize()
+    for k in range(S):
+        sel, c, score, acc = zo.search_levels(loss.numpy(), base.numpy(), time.numpy(), n_opt.numpy(),
+                                              objective.numpy(), coef0[k].numpy(), float(budgets[k]),
+                                              n_buckets, mask[k].numpy(), values[k].numpy())
+        assert int(out["status"][k]) == 0
+        assert out["selected"][k].tolist() == sel
+        assert int(out["n_accepted"][k]) == acc
+        assert np.array_equal(out["coef"][k].cpu().numpy(), c)
+        assert float(out["objective"][k]) == score
+    # no steps: the selection of coef0 itself
+    out0 = z.search_levels(loss.cuda(), base.cuda(), time.cuda(), n_opt.cuda(), objective.cuda(),
+                           coef0.cuda(), budgets.cuda(), n_buckets, mask[:, :0].contiguous().cuda(),
+                           values[:, :0].contiguous().cuda())
+    ref = z.select_levels(loss.cuda(), base.cuda(), time.cuda(), n_opt.cuda(), coef0[:1].cuda(),
+                          float(budgets[1]), n_buckets)
+    assert out0["selected"][1].tolist() == ref["selected"][0].tolist()
+    assert out0["n_accepted"].tolist() == [0, 0, 0]

@@ -565,3 +565,37 @@ def test_level_selection_limits_and_monotonicity():
     time3[np.arange(6), n_opt - 1] = 1.0
     assert zo.select_levels(loss, base, time3, n_opt, coef, 5.9, 60)[0] is None
     assert zo.select_levels(loss, base, time3, n_opt, coef, 6.0, 60)[0] == [int(k) - 1 for k in n_opt]
+
+
+def test_mutation_search_pins():
+    """No marks: nothing is ever accepted and the result is coef0's selection.  If the score is
+    the cost under some coefficients c* and one step sets all coefficients to c*, that step's
+    selection is optimal among everything that fits, so it is accepted (unless coef0 already
+    reached that score) and no later mutation can be: final score = the optimum of c*."""
+    rng = np.random.default_rng(5)
+    n_mod, max_opt, n_buckets, steps = 6, 5, 120, 12
+    loss, base, time, n_opt = random_database(rng, n_mod, max_opt)
+    budget = 0.4 * float(time[:, 0].sum())
+    coef0 = rng.uniform(0.1, 3.0, size=n_mod).astype(np.float32)
+    c_star = rng.uniform(0.1, 3.0, size=n_mod).astype(np.float32)
+    objective = (c_star[:, None].astype(np.float64) * (loss.astype(np.float64) / base[:, None])).astype(np.float32)
+    values = rng.uniform(0.1, 3.0, size=(steps, n_mod)).astype(np.float32)
+    none = np.zeros((steps, n_mod), np.uint8)
+    sel0, _, _ = zo.select_levels(loss, base, time, n_opt, coef0, budget, n_buckets)
+    score0 = sum(float(objective[m, s]) for m, s in enumerate(sel0))
+    sel, c, score, acc = zo.search_levels(loss, base, time, n_opt, objective, coef0, budget, n_buckets,
+                                          none, values)
+    assert sel == sel0 and acc == 0 and np.array_equal(c, coef0) and np.isclose(score, score0)
+    mask = (rng.uniform(size=(steps, n_mod)) < 0.3).astype(np.uint8)
+    mask[3] = 1
+    values[3] = c_star
+    sel_star, cost_star, _ = zo.select_levels(loss, base, time, n_opt, c_star, budget, n_buckets)
+    sel, c, score, acc = zo.search_levels(loss, base, time, n_opt, objective, coef0, budget, n_buckets,
+                                          mask, values)
+    assert np.isclose(score, cost_star, rtol=1e-6)        # objective was rounded to fp32
+    t_sel = sum(float(time[m, s]) for m, s in enumerate(sel))
+    assert t_sel <= budget
+    # the score never goes up as steps are added
+    scores = [zo.search_levels(loss, base, time, n_opt, objective, coef0, budget, n_buckets,
+                               mask[:t], values[:t])[2] for t in range(steps + 1)]
+    assert all(a >= b for a, b in zip(scores, scores[1:])) and np.isclose(scores[0], score0)
