@@ -390,7 +390,7 @@ def run_ours(args, shape):
     # ---- the Hessian from token-major activations (one token per row, the layout a forward pass
     # emits): one call on the whole calibration set, and eight calibration batches with beta = 1
     tok = None
-    if not args.skip_stream_leg:
+    if not args.skip_extras:
         A = X.transpose(1, 2).contiguous()
         Ht = torch.empty_like(H)
         t_ws = torch.empty(z.hessian_tokens_workspace_bytes(L, d, N, 0) + 256, dtype=torch.uint8,
@@ -428,7 +428,7 @@ def run_ours(args, shape):
     # ---- reshaping the whole database: survivors, compacted snapshot and compacted previous layer
     # (a stand-in FC1 of shape [d, r]) for every level
     reshape = None
-    if not args.skip_stream_leg:
+    if not args.skip_extras:
         prev = torch.randn(L, d, r, device=dev)
 
         def reshape_all():
@@ -459,7 +459,7 @@ def run_ours(args, shape):
     # 12 FFN), the paper's level grid, 10^4 time buckets; 1024 coefficient vectors per launch, and
     # the 1000-step mutation search for 148 speedup targets at once (one CTA each)
     select = None
-    if not args.skip_stream_leg:
+    if not args.skip_extras:
         gsel = torch.Generator().manual_seed(1)
         grids = [wl.paper_level_grid(12, 64), wl.paper_level_grid(G, 1)]
         max_opt = 1 + max(len(x) for x in grids)
@@ -631,6 +631,8 @@ def main():
     ap.add_argument("--max-removed", type=int, default=0,
                     help="profiling aid: stop the greedy loop after this many removals")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling aid: no host-buffer leg")
+    ap.add_argument("--skip-extras", action="store_true",
+                    help="profiling aid: no token-major Hessian / reshaping / level-selection legs")
     ap.add_argument("--skip-stream-leg", action="store_true",
                     help="profiling aid: do not time the per-step streaming variant")
     args = ap.parse_args()

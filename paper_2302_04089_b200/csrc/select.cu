@@ -20,7 +20,7 @@
 namespace ziplm {
 namespace {
 
-constexpr int SEL_THREADS = 512;
+constexpr int SEL_THREADS = 1024;
 constexpr int SEL_MAX_OPT = 255;          // options per module (argmin stored in a byte)
 constexpr int SEL_MAX_BUCKETS = 12000;    // two float64 rows of n_buckets + 1 fit shared memory
 constexpr int SEL_MAX_MOD = 512;          // modules per search (coefficient vectors in shared memory)
@@ -50,17 +50,31 @@ __device__ void dp_solve(const float* __restrict__ loss, const float* __restrict
             if (s_cost[s] != s_cost[s] || u != u) *nonfinite = 1;
         }
         __syncthreads();
-        for (int b = tid; b <= n_buckets; b += SEL_THREADS) {
-            double best = inf;
-            int arg = 0;
+        // four buckets per thread and pass, so that an option's units and cost are fetched once
+        // for four evaluations
+        for (int b0 = tid; b0 <= n_buckets; b0 += 4 * SEL_THREADS) {
+            double best[4] = {inf, inf, inf, inf};
+            int arg[4] = {0, 0, 0, 0};
             for (int s = 0; s < no; ++s) {
                 const int u = s_units[s];
-                if (u > b) continue;
-                const double v = f0[b - u] + s_cost[s];
-                if (v < best) { best = v; arg = s; }
+                const double c = s_cost[s];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int b = b0 + j * SEL_THREADS;
+                    if (b <= n_buckets && u <= b) {
+                        const double v = f0[b - u] + c;
+                        if (v < best[j]) { best[j] = v; arg[j] = s; }
+                    }
+                }
             }
-            f1[b] = best;
-            ch[(size_t)m * (n_buckets + 1) + b] = (unsigned char)arg;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int b = b0 + j * SEL_THREADS;
+                if (b <= n_buckets) {
+                    f1[b] = best[j];
+                    ch[(size_t)m * (n_buckets + 1) + b] = (unsigned char)arg[j];
+                }
+            }
         }
         double* t = f0; f0 = f1; f1 = t;
     }
