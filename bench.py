@@ -552,7 +552,7 @@ def run_ours(args, shape):
             phases_ms={k: round(v[0], 3) for k, v in phases.items() if v[1] > 0},
             phases_note="per-phase CUDA-event times of one extra step with the layer groups run "
                         f"back to back (that step: {ms_one_group:.1f} ms); the timed steps overlap "
-                        "four layer groups on internal streams",
+                        "six layer groups on internal streams",
             e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                      ms_per_step=ms_e2e, steps=e2e_steps, single_batch_ms=ms_e2e_single,
                      note="a stream of batches through the public calls: every step uploads its own "

@@ -748,8 +748,24 @@ ziplm_status factor_range(const InvCtx& c, int lo, int hi) {
             k_factor_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmallSmem));
         if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
         PhaseScope ps(PH_INV_LEAVES, c.st);
-        k_factor_small<<<c.L, kSmallThreads, sizeof(SmallSmem), c.st>>>(c.A, c.F, c.M, c.dp, lo, hi - lo,
-                                                              c.layer_status);
+        // One CTA per layer and a long dependent chain: launched at the highest priority, so that
+        // it does not queue behind the wide kernels of other layer groups.
+        static int prio = [] {
+            int least = 0, greatest = 0;
+            return cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess ? greatest : 0;
+        }();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(c.L);
+        cfg.blockDim = dim3(kSmallThreads);
+        cfg.dynamicSmemBytes = sizeof(SmallSmem);
+        cfg.stream = c.st;
+        cudaLaunchAttribute la[1];
+        la[0].id = cudaLaunchAttributePriority;
+        la[0].val.priority = prio;
+        cfg.attrs = la;
+        cfg.numAttrs = 1;
+        ZIPLM_CHECK_CUDA(cudaLaunchKernelEx(&cfg, k_factor_small, c.A, c.F, c.M, c.dp, lo, hi - lo,
+                                            c.layer_status));
         ZIPLM_CHECK_LAUNCH();
         return ZIPLM_OK;
     }

@@ -837,6 +837,10 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
     };
 
     int n = G, slot = 0, t = 0;
+    int prio_least = 0, prio_greatest = 0;
+    ZIPLM_CHECK_CUDA(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
+    const char* prio_env = getenv("ZIPLM_STEPS_PRIORITY");
+    const int steps_priority = (prio_env && prio_env[0] == '0') ? prio_least : prio_greatest;
     // rank-32 update of H^-1 and Q: the fp32 FMA kernel by default, which is the faster one so far
     const char* upd_env = getenv("ZIPLM_LAZY_UPDATE");
     const bool use_tc = upd_env && upd_env[0] == 't';   // "tc": tcgen05 variant (prune_lazy_tc.cu)
@@ -862,13 +866,18 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
             cfg.blockDim = dim3(STEP_THREADS);
             cfg.dynamicSmemBytes = (size_t)2 * BMAX * S * sizeof(float);
             cfg.stream = st;
-            cudaLaunchAttribute attr[1];
+            cudaLaunchAttribute attr[2];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = cs;
             attr[0].val.clusterDim.y = 1;
             attr[0].val.clusterDim.z = 1;
+            // The steps kernel is the latency chain of a layer group and needs whole SMs for its
+            // clusters: at the highest launch priority its CTAs go ahead of the queued CTAs of the
+            // other groups' wide update kernels as SMs drain.
+            attr[1].id = cudaLaunchAttributePriority;
+            attr[1].val.priority = steps_priority;
             cfg.attrs = attr;
-            cfg.numAttrs = 1;
+            cfg.numAttrs = 2;
             ZIPLM_CHECK_CUDA(cudaLaunchKernelEx(
                 &cfg, k_lazy_steps, n, S, t, nsteps, d, G, r, rp, (const float*)w.A[cur],
                 (const float*)w.Q[cur], (const float*)w.Wt[cur], (const double*)w.dA[cur],

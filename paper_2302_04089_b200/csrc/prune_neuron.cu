@@ -389,7 +389,7 @@ static bool use_lazy_path(int d) {
 // they are split into groups that run the whole pipeline on streams of their own: one group's
 // latency-bound kernels then overlap the other groups' bandwidth- and ALU-bound ones.
 constexpr int kMaxGroups = 8;
-constexpr int kDefaultGroups = 4;
+constexpr int kDefaultGroups = 6;
 
 static int layer_groups(int L) {
     int g = kDefaultGroups;
