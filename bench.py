@@ -180,9 +180,10 @@ NCU_TRAFFIC = {
     # k_dgemm_tiles, top-level product F21 = A21 M11^T: profiles/inverse_kernels_c3.md
     "k_dgemm_tiles": dict(bytes=3 * (116.6e6 + 49.0e6), launch="F21 = A21 M11^T, 12 x 24 macro tiles",
                           algorithmic=None),
-    # k_neuron_update at n = 3066: profiles/k_neuron_update_c3_4layers.md
-    "k_neuron_update": dict(bytes=3 * (113.8e6 + 56.6e6), launch="n = 3066",
-                            algorithmic=12 * (8.0 * 768 * 3066 + 4.0 * 3066 * 3066)),
+    # k_neuron_update, first step at full size (12 layers, n = 3071):
+    # profiles/k_neuron_update_c3_12layers_every_step.md
+    "k_neuron_update": dict(bytes=343.1e6 + 281.9e6, launch="n = 3071, 12 layers",
+                            algorithmic=12 * (8.0 * 768 * 3071 + 4.0 * 3071 * 3071)),
 }
 
 
