@@ -174,8 +174,9 @@ LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in p
 # proportion to the layers).  Only valid for the bench workload; the kernels have not changed
 # since the captures.
 NCU_TRAFFIC = {
-    # k_lazy_update_aq, first block (n_new = 3040): profiles/k_lazy_kernels_c3_4layers.md
-    "k_lazy_update_aq": dict(bytes=3 * (169.8e6 + 235.8e6), launch="n_new = 3040, m = 32",
+    # k_lazy_update_aq, first block at full size (12 layers, n_new = 3040):
+    # profiles/k_lazy_update_aq_c3_12layers_every_launch.md
+    "k_lazy_update_aq": dict(bytes=523.1e6 + 826.2e6, launch="n_new = 3040, m = 32, 12 layers",
                              algorithmic=12 * 24.0 * 3040 * 3039 / 2),
     # k_dgemm_tiles, top-level product F21 = A21 M11^T: profiles/inverse_kernels_c3.md
     "k_dgemm_tiles": dict(bytes=3 * (116.6e6 + 49.0e6), launch="F21 = A21 M11^T, 12 x 24 macro tiles",
