@@ -46,7 +46,7 @@ typedef enum {
     ZIPLM_ERR_UNSUPPORTED = 7  /* valid request outside what this build implements            */
 } ziplm_status;
 
-typedef enum { ZIPLM_F32 = 0, ZIPLM_BF16 = 1 } ziplm_dtype;
+typedef enum { ZIPLM_F32 = 0, ZIPLM_BF16 = 1, ZIPLM_F16 = 2 } ziplm_dtype;
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* ziplm_status_string(ziplm_status s);
@@ -58,7 +58,8 @@ const char* ziplm_status_string(ziplm_status s);
  *
  * alpha = 2 gives the paper's Hessian; beta = 1 adds one more batch of tokens to a running sum,
  * beta = 0 overwrites.  Products are accumulated in fp32; fp32 inputs keep fp32 accuracy (on the
- * tensor-core route they are split into TF32 terms), bf16 inputs are multiplied exactly.
+ * tensor-core route they are split into TF32 terms), bf16 and fp16 inputs are multiplied exactly
+ * (an fp16 or bf16 product has at most 22 significant bits).
  *
  *   H          dev, [L, d, d] fp32, in/out; full symmetric matrix on return
  *   X          dev, [L, d, ldx] of x_dtype, token index contiguous; only the first n_tokens

@@ -29,7 +29,8 @@ class Status(enum.IntEnum):
     ERR_UNSUPPORTED = 7
 
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
+_DTYPES = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}
 
 
 class ZiplmError(RuntimeError):
@@ -151,17 +152,17 @@ def prune_workspace_bytes(L: int, d_row: int, d_col: int, group_size: int, n_lev
 
 def hessian_accumulate(X: torch.Tensor, H: Optional[torch.Tensor] = None, alpha: float = 2.0,
                        beta: float = 0.0, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """H = beta * H + alpha * X X^T per layer.  X [L, d, N] fp32 or bf16 (tokens contiguous)."""
+    """H = beta * H + alpha * X X^T per layer.  X [L, d, N] fp32, bf16 or fp16 (tokens contiguous)."""
     lib = load_library()
     if X.dim() != 3 or not X.is_cuda or X.stride(2) != 1 and X.shape[2] > 1:
         raise ValueError("X must be a CUDA tensor [L, d, N] with contiguous tokens")
-    if X.dtype not in (torch.float32, torch.bfloat16):
-        raise ValueError("X must be fp32 or bf16")
+    if X.dtype not in _DTYPES:
+        raise ValueError("X must be fp32, bf16 or fp16")
     L, d, N = X.shape
     if X.stride(0) != d * X.stride(1):
         raise ValueError("layers of X must be evenly pitched")
     ldx = X.stride(1) if N > 0 else max(N, 1)
-    dt = F32 if X.dtype == torch.float32 else BF16
+    dt = _DTYPES[X.dtype]
     if H is None:
         H = torch.zeros(L, d, d, dtype=torch.float32, device=X.device)
         beta = 0.0
@@ -180,18 +181,18 @@ def hessian_accumulate(X: torch.Tensor, H: Optional[torch.Tensor] = None, alpha:
 def hessian_accumulate_tokens(A: torch.Tensor, H: Optional[torch.Tensor] = None, alpha: float = 2.0,
                               beta: float = 0.0,
                               workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """H = beta * H + alpha * A^T A per layer.  A [L, N, d] fp32 or bf16, one token per row
+    """H = beta * H + alpha * A^T A per layer.  A [L, N, d] fp32, bf16 or fp16, one token per row
     (features contiguous); the row pitch may exceed d.  See ziplm_hessian_accumulate_tokens."""
     lib = load_library()
     if A.dim() != 3 or not A.is_cuda or A.stride(2) != 1 and A.shape[2] > 1:
         raise ValueError("A must be a CUDA tensor [L, N, d] with contiguous features")
-    if A.dtype not in (torch.float32, torch.bfloat16):
-        raise ValueError("A must be fp32 or bf16")
+    if A.dtype not in _DTYPES:
+        raise ValueError("A must be fp32, bf16 or fp16")
     L, N, d = A.shape
     lda = A.stride(1) if N > 1 else d
     if L > 1 and N > 0 and A.stride(0) != N * lda:
         raise ValueError("layers of A must be evenly pitched")
-    dt = F32 if A.dtype == torch.float32 else BF16
+    dt = _DTYPES[A.dtype]
     if H is None:
         H = torch.zeros(L, d, d, dtype=torch.float32, device=A.device)
         beta = 0.0

@@ -50,7 +50,7 @@ ziplm_status ziplm_hessian_accumulate(float* H, const void* X, ziplm_dtype x_dty
                                       long long n_tokens, long long ldx, float alpha, float beta,
                                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (L < 1 || d < 1 || n_tokens < 0 || ldx < n_tokens || !H) return ZIPLM_ERR_INVALID_ARG;
-    if (x_dtype != ZIPLM_F32 && x_dtype != ZIPLM_BF16) return ZIPLM_ERR_INVALID_ARG;
+    if (x_dtype != ZIPLM_F32 && x_dtype != ZIPLM_BF16 && x_dtype != ZIPLM_F16) return ZIPLM_ERR_INVALID_ARG;
     if (!(beta == 0.f || beta == 1.f) || !isfinite(alpha)) return ZIPLM_ERR_INVALID_ARG;
     const size_t esz = (x_dtype == ZIPLM_F32) ? 4 : 2;
     if (n_tokens > 0) {
@@ -75,7 +75,7 @@ ziplm_status ziplm_hessian_accumulate_tokens(float* H, const void* A, ziplm_dtyp
                                              float beta, void* workspace, size_t workspace_bytes,
                                              void* cuda_stream) {
     if (L < 1 || d < 1 || n_tokens < 0 || lda < d || !H) return ZIPLM_ERR_INVALID_ARG;
-    if (a_dtype != ZIPLM_F32 && a_dtype != ZIPLM_BF16) return ZIPLM_ERR_INVALID_ARG;
+    if (a_dtype != ZIPLM_F32 && a_dtype != ZIPLM_BF16 && a_dtype != ZIPLM_F16) return ZIPLM_ERR_INVALID_ARG;
     if (!(beta == 0.f || beta == 1.f) || !isfinite(alpha)) return ZIPLM_ERR_INVALID_ARG;
     const size_t esz = (a_dtype == ZIPLM_F32) ? 4 : 2;
     if (n_tokens > 0 && (!A || !aligned(A, esz))) return ZIPLM_ERR_INVALID_ARG;

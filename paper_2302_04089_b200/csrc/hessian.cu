@@ -9,6 +9,7 @@
 // tensor-core route (hessian_tc.cu) is the default; the CUDA-core route serves token counts
 // below one K block and can be forced with ZIPLM_HESSIAN_ROUTE=simt for comparison.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -36,12 +37,21 @@ __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16* p, flo
     v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
 }
 
+template <>
+__device__ __forceinline__ void load4<__half>(const __half* p, float (&v)[4]) {
+    const uint2 t = *reinterpret_cast<const uint2*>(p);
+    const __half2 a = *reinterpret_cast<const __half2*>(&t.x), b = *reinterpret_cast<const __half2*>(&t.y);
+    v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b);
+}
+
 template <typename T>
 __device__ __forceinline__ float to_f32(T v);
 template <>
 __device__ __forceinline__ float to_f32<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <>
+__device__ __forceinline__ float to_f32<__half>(__half v) { return __half2float(v); }
 
 // TOK: the input is token-major, [N, ldx] per layer with the feature index contiguous; element
 // (feature i, token k) then sits at k * ldx + i and is fetched with scalar loads.
@@ -158,14 +168,19 @@ ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, bool token_maj
     const dim3 grid(T * (T + 1) / 2, L);
     const float* Xf = static_cast<const float*>(X);
     const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
+    const __half* Xh = static_cast<const __half*>(X);
     if (dt == ZIPLM_F32 && !token_major)
         k_syrk_simt<float, false><<<grid, 256, 0, st>>>(H, Xf, d, N, ldx, alpha, beta);
     else if (dt == ZIPLM_F32)
         k_syrk_simt<float, true><<<grid, 256, 0, st>>>(H, Xf, d, N, ldx, alpha, beta);
-    else if (!token_major)
+    else if (dt == ZIPLM_BF16 && !token_major)
         k_syrk_simt<__nv_bfloat16, false><<<grid, 256, 0, st>>>(H, Xb, d, N, ldx, alpha, beta);
-    else
+    else if (dt == ZIPLM_BF16)
         k_syrk_simt<__nv_bfloat16, true><<<grid, 256, 0, st>>>(H, Xb, d, N, ldx, alpha, beta);
+    else if (!token_major)
+        k_syrk_simt<__half, false><<<grid, 256, 0, st>>>(H, Xh, d, N, ldx, alpha, beta);
+    else
+        k_syrk_simt<__half, true><<<grid, 256, 0, st>>>(H, Xh, d, N, ldx, alpha, beta);
     ZIPLM_CHECK_LAUNCH();
     return ZIPLM_OK;
 }

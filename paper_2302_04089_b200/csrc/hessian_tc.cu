@@ -6,7 +6,8 @@
 // tensor map serves A and B.  Only the 128 x 128 tiles on or below the diagonal are computed; an
 // off-diagonal tile is stored twice (as is, and transposed).
 //
-//   bf16 X : kind::f16 (bf16 x bf16, exact products, fp32 accumulate), K block of 64 tokens.
+//   bf16 / fp16 X : kind::f16 (both operands of the same 16-bit type, exact products, fp32
+//            accumulate), K block of 64 tokens.
 //   fp32 X : a pre-pass writes X_hi (fp32 with the 13 low mantissa bits cleared = a TF32 value)
 //            and X_lo = X - X_hi; the kernel accumulates hi*hi + hi*lo + lo*hi with kind::tf32,
 //            which keeps ~21 mantissa bits per product.  K block of 32 tokens.
@@ -51,7 +52,7 @@ template <bool TF32>
 __global__ void __launch_bounds__(THREADS, 1)
 k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
           float* __restrict__ H, int d, int num_kb, float alpha, float beta, int layer0,
-          int* __restrict__ err_word) {
+          int* __restrict__ err_word, uint32_t fmt16) {
     using C = Cfg<TF32>;
     constexpr int STAGE_BYTES = C::TILES * TILE_BYTES;
     constexpr uint32_t TMEM_COLS = TF32 ? 512u : 256u;   // main x2 (+ cross terms), power of two
@@ -118,7 +119,8 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- MMA issuer
-            constexpr uint32_t idesc = make_idesc(TF32 ? 2u : 1u, TM, TM);
+            // operand format of the instruction: 2 = TF32; 16-bit inputs: 1 = BF16, 0 = F16 (A and B alike)
+            const uint32_t idesc = make_idesc(TF32 ? 2u : fmt16, TM, TM);
             const uint32_t tmem_cross = tmem_base + 256u;
             int kb = 0;
             for (int c = 0; c < num_chunks && !failed; ++c) {
@@ -366,8 +368,9 @@ bool quad_rows(const void* A, long long lda, size_t esz) {
 
 // 3-D map over [layers, rows, K] with box {128 bytes of K, 128 rows, 1 layer}, 128-byte swizzle,
 // zero fill outside the tensor (ragged d and ragged token counts contribute zeros).
-bool make_map(CUtensorMap* m, const void* base, bool f32, long long K, int rows, int layers,
+bool make_map(CUtensorMap* m, const void* base, ziplm_dtype dt, long long K, int rows, int layers,
               long long pitch_elems) {
+    const bool f32 = (dt == ZIPLM_F32);
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     const size_t esz = f32 ? 4 : 2;
@@ -375,7 +378,8 @@ bool make_map(CUtensorMap* m, const void* base, bool f32, long long K, int rows,
     cuuint64_t strides[2] = {(cuuint64_t)pitch_elems * esz, (cuuint64_t)pitch_elems * esz * rows};
     cuuint32_t box[3] = {(cuuint32_t)(ROW_BYTES / esz), (cuuint32_t)TM, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+    CUresult r = enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                            : dt == ZIPLM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
                      const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -422,6 +426,7 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
                             size_t ws_bytes, cudaStream_t st) {
     if (ws_bytes < hessian_tc_workspace_bytes(L, d, N, dt, token_major)) return ZIPLM_ERR_WORKSPACE;
     const bool f32 = (dt == ZIPLM_F32);
+    const uint32_t fmt16 = (dt == ZIPLM_F16) ? 0u : 1u;
     Carver c(ws);
     int* err_word = c.take<int>(1);
     ZIPLM_CHECK_CUDA(cudaMemsetAsync(err_word, 0, sizeof(int), st));
@@ -473,10 +478,10 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
                 }
             }
             CUtensorMap mh, ml;
-            if (!make_map(&mh, hi, true, N, d, ln, np) || !make_map(&ml, lo, true, N, d, ln, np))
+            if (!make_map(&mh, hi, ZIPLM_F32, N, d, ln, np) || !make_map(&ml, lo, ZIPLM_F32, N, d, ln, np))
                 return ZIPLM_ERR_CUDA;
             k_syrk_tc<true><<<dim3(n_tiles, ln), THREADS, smem_tf32, st>>>(mh, ml, H, d, num_kb, alpha, beta,
-                                                                      l0, err_word);
+                                                                      l0, err_word, 2u);
             ZIPLM_CHECK_LAUNCH();
         }
     } else if (token_major) {
@@ -498,9 +503,9 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
                         Ac, ldx, N, d, np, xt, nullptr);
             ZIPLM_CHECK_LAUNCH();
             CUtensorMap mx;
-            if (!make_map(&mx, xt, false, N, d, ln, np)) return ZIPLM_ERR_CUDA;
+            if (!make_map(&mx, xt, dt, N, d, ln, np)) return ZIPLM_ERR_CUDA;
             k_syrk_tc<false><<<dim3(n_tiles, ln), THREADS, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
-                                                                       l0, err_word);
+                                                                       l0, err_word, fmt16);
             ZIPLM_CHECK_LAUNCH();
         }
     } else {
@@ -511,9 +516,9 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
             const int ln = (L - l0 < 65535) ? (L - l0) : 65535;
             CUtensorMap mx;
             const __nv_bfloat16* Xc = static_cast<const __nv_bfloat16*>(X) + (size_t)l0 * d * ldx;
-            if (!make_map(&mx, Xc, false, N, d, ln, ldx)) return ZIPLM_ERR_CUDA;
+            if (!make_map(&mx, Xc, dt, N, d, ln, ldx)) return ZIPLM_ERR_CUDA;
             k_syrk_tc<false><<<dim3(n_tiles, ln), THREADS, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
-                                                                       l0, err_word);
+                                                                       l0, err_word, fmt16);
             ZIPLM_CHECK_LAUNCH();
         }
     }

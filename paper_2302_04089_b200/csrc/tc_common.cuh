@@ -103,7 +103,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
 }
 
 // Instruction descriptor: fp32 accumulate, A and B K-major, M x N output tile; operand format
-// 2 = TF32 or 1 = BF16.
+// 2 = TF32 (kind::tf32); 1 = BF16 or 0 = F16 (kind::f16, A and B of the same type).
 __host__ __device__ constexpr uint32_t make_idesc(uint32_t fmt, int M, int N) {
     return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(N >> 3) << 17) |
            ((uint32_t)(M >> 4) << 24);

@@ -36,7 +36,7 @@ def run_case(shape, levels=None, layers=None, check_layers=None, base=True):
 
 
 # ------------------------------------------------------------------ Hessian (a1)
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("d,N,ldx", [(64, 256, 256), (200, 1000, 1000), (130, 77 * 8, 640), (96, 8, 8)])
 def test_hessian_matches_oracle(dtype, d, N, ldx):
     z = zb()
@@ -84,7 +84,7 @@ def token_major_case(dtype, d, N, lda, L=2):
     return X, A
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("d,N,lda", [(64, 256, 64), (200, 1000, 208), (130, 613, 131), (96, 8, 96),
                                      (33, 31, 40), (257, 4099, 257), (130, 613, 132), (257, 4099, 260)])
 def test_hessian_from_token_major_activations_matches_oracle(dtype, d, N, lda):
@@ -105,7 +105,7 @@ def test_hessian_from_token_major_activations_matches_oracle(dtype, d, N, lda):
         assert torch.equal(H, z.hessian_accumulate(X.cuda()))
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 def test_hessian_streamed_batch_by_batch(dtype):
     """beta = 1 over ragged calibration batches (one of them shorter than a K block, one empty)
     against the oracle's sum of outer products over all tokens."""

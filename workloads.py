@@ -38,7 +38,7 @@ class LayerShape:
     group_size: int      # g: 1 = FFN neuron, 64 = attention head
     levels: Tuple[int, ...]  # remaining-structure counts, strictly decreasing
     d_latent: int = 0    # ffn recipe: width of the pre-activation sources
-    x_dtype: str = "f32"  # "f32" or "bf16"
+    x_dtype: str = "f32"  # "f32", "bf16" or "f16"
     seed_base: int = 0
     damp_frac: float = 0.01
 
@@ -143,6 +143,8 @@ def make_activations(shape: LayerShape, layer: int, device: str = "cpu",
         raise ValueError(f"unknown recipe {shape.recipe!r}")
     if shape.x_dtype == "bf16":
         X = X.to(torch.bfloat16)
+    elif shape.x_dtype == "f16":
+        X = X.to(torch.float16)
     return X.contiguous()
 
 
