@@ -448,6 +448,10 @@ static ziplm_status run_prune_lazy_grouped(const float* W, const float* H, int L
         return run_prune_lazy(W, H, L, r, d, damp_frac, levels, n_levels, W_snap, loss, base_loss,
                               order, saliency, layer_status, ws,
                               lazy_workspace_bytes(L, r, d, n_levels), st);
+    // Calls take consecutive streams of the pool in turn, so that two calls that the caller runs
+    // concurrently (different layers on different streams) do not queue behind each other.
+    static std::atomic<unsigned> next_stream{0};
+    const unsigned first = next_stream.fetch_add((unsigned)groups);
     cudaEvent_t fork, join[kMaxGroups];
     ZIPLM_CHECK_CUDA(cudaEventCreateWithFlags(&fork, cudaEventDisableTiming));
     ZIPLM_CHECK_CUDA(cudaEventRecord(fork, st));
@@ -456,7 +460,7 @@ static ziplm_status run_prune_lazy_grouped(const float* W, const float* H, int L
     for (int g = 0; g < groups; ++g) {
         const int l0 = group_begin(L, groups, g), Lg = group_begin(L, groups, g + 1) - l0;
         const size_t bytes = lazy_workspace_bytes(Lg, r, d, n_levels);
-        cudaStream_t sg = pool[g];
+        cudaStream_t sg = pool[(first + (unsigned)g) % kMaxGroups];
         bool ok = cudaStreamWaitEvent(sg, fork, 0) == cudaSuccess;
         if (ok && rc == ZIPLM_OK)
             rc = run_prune_lazy(W + (size_t)l0 * r * d, H + (size_t)l0 * d * d, Lg, r, d, damp_frac,
