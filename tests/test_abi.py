@@ -24,7 +24,11 @@ def test_header_declares_the_expected_entry_points():
     syms = declared_symbols()
     for name in ("ziplm_hessian_accumulate", "ziplm_prune_layers", "ziplm_damped_inverse",
                  "ziplm_hessian_workspace_bytes", "ziplm_prune_workspace_bytes",
-                 "ziplm_inverse_workspace_bytes", "ziplm_status_string"):
+                 "ziplm_inverse_workspace_bytes", "ziplm_status_string",
+                 "ziplm_hessian_accumulate_tokens", "ziplm_hessian_tokens_workspace_bytes",
+                 "ziplm_kept_structures", "ziplm_gather_columns", "ziplm_gather_rows",
+                 "ziplm_select_levels", "ziplm_select_workspace_bytes", "ziplm_search_levels",
+                 "ziplm_search_workspace_bytes", "ziplm_damped_inverse_noalloc"):
         assert name in syms
 
 
@@ -44,6 +48,11 @@ def test_status_strings_and_workspace_queries(lib):
     assert 0 < a < b and a % 256 == 0 and b % 256 == 0
     assert lib.ziplm_prune_workspace_bytes(1, 64, 255, 64, 3) == 0     # 255 % 64 != 0
     assert lib.ziplm_inverse_workspace_bytes(2, 100) >= 2 * 2 * 128 * 128 * 8
+    lib.ziplm_select_workspace_bytes.restype = ctypes.c_size_t
+    lib.ziplm_search_workspace_bytes.restype = ctypes.c_size_t
+    assert lib.ziplm_select_workspace_bytes(3, 24, 10000) >= 3 * 24 * 10001
+    assert lib.ziplm_search_workspace_bytes(3, 24, 10000) > lib.ziplm_select_workspace_bytes(3, 24, 10000)
+    assert lib.ziplm_select_workspace_bytes(0, 24, 10000) == 0
 
 
 def test_binding_mirrors_the_abi_names():
