@@ -28,20 +28,11 @@
 #include <cooperative_groups.h>
 #include <math.h>
 
-#include <cuda.h>
 #include <stdlib.h>
 
 #include "common.cuh"
 
 namespace ziplm {
-
-// Tensor-core rank-32 update of H^-1 and Q (prune_lazy_tc.cu).
-size_t lazy_tc_pack_floats(int L, int d);
-bool lazy_tc_make_map(CUtensorMap* m, const float* P, int L, int d);
-ziplm_status run_lazy_update_aq_tc(const CUtensorMap& map, int L, int n_new, int m, int d,
-                                   const float* A, const float* Q, float* A2, float* Q2,
-                                   const int* src, const float* U, const float* Z, float* P,
-                                   int* layer_status, cudaStream_t st);
 
 namespace {
 
@@ -740,7 +731,6 @@ struct LazyWs {
     float* A[2]; float* Q[2]; float* Wt[2];
     double* dA[2]; double* dQ[2]; int* idx[2];
     int* src; int* pos_of; float* U; float* Z; float* C;
-    float* P;                          // packed split operands of the tensor-core update
     LazyState* state; double* lam; double* base_acc;
     void* aux; size_t aux_bytes;       // shared by the inverse and by the Gram-matrix product
     int rp; size_t total;
@@ -761,7 +751,6 @@ LazyWs carve_lazy(void* ws, int L, int r, int d) {
     w.U = c.take<float>((size_t)L * BMAX * d);
     w.Z = c.take<float>((size_t)L * BMAX * d);
     w.C = c.take<float>((size_t)L * BMAX * w.rp);
-    w.P = c.take<float>(lazy_tc_pack_floats(L, d));
     w.state = c.take<LazyState>((size_t)L);
     w.lam = c.take<double>((size_t)L);
     w.base_acc = c.take<double>((size_t)L);
@@ -839,13 +828,7 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
     int n = G, slot = 0, t = 0;
     int prio_least = 0, prio_greatest = 0;
     ZIPLM_CHECK_CUDA(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
-    const char* prio_env = getenv("ZIPLM_STEPS_PRIORITY");
-    const int steps_priority = (prio_env && prio_env[0] == '0') ? prio_least : prio_greatest;
-    // rank-32 update of H^-1 and Q: the fp32 FMA kernel by default, which is the faster one so far
-    const char* upd_env = getenv("ZIPLM_LAZY_UPDATE");
-    const bool use_tc = upd_env && upd_env[0] == 't';   // "tc": tcgen05 variant (prune_lazy_tc.cu)
-    CUtensorMap map;
-    if (use_tc && !lazy_tc_make_map(&map, w.P, L, d)) return ZIPLM_ERR_CUDA;
+    const int steps_priority = prio_greatest;
     if (slot < n_levels && levels[slot] == n) {
         s = snapshot(n, slot++);
         if (s != ZIPLM_OK) return s;
@@ -895,19 +878,12 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
                 n_new, nsteps, d, rp, w.Wt[cur], w.Wt[nxt], w.src, w.U, w.C);
             ZIPLM_CHECK_LAUNCH();
         }
-        if (n_new > 1 && use_tc) {
+        if (n_new > 1) {
             PhaseScope ps(PH_LAZY_UPDATE_AQ, st);
-            s = run_lazy_update_aq_tc(map, L, n_new, nsteps, d, w.A[cur], w.Q[cur], w.A[nxt], w.Q[nxt],
-                                      w.src, w.U, w.Z, w.P, layer_status, st);
-            if (s != ZIPLM_OK) return s;
-        } else if (n_new > 1) {
-            PhaseScope ps(PH_LAZY_UPDATE_AQ, st);
-            {
-                const int T = (n_new + 63) / 64;
-                k_lazy_update_aq<<<dim3(T * (T + 1) / 2, L), 128, 0, st>>>(
-                    n_new, nsteps, d, w.A[cur], w.Q[cur], w.A[nxt], w.Q[nxt], w.src, w.U, w.Z);
-                ZIPLM_CHECK_LAUNCH();
-            }
+            const int T = (n_new + 63) / 64;
+            k_lazy_update_aq<<<dim3(T * (T + 1) / 2, L), 128, 0, st>>>(
+                n_new, nsteps, d, w.A[cur], w.Q[cur], w.A[nxt], w.Q[nxt], w.src, w.U, w.Z);
+            ZIPLM_CHECK_LAUNCH();
         }
         cur = nxt;
         n = n_new;

@@ -127,12 +127,10 @@ def lockstep_head(W, H32, shape, out, layer, n_steps):
     return near
 
 
-@pytest.mark.parametrize("path", ["lazy", "lazy_tc", "stream"])
+@pytest.mark.parametrize("path", ["lazy", "stream"])
 def test_c3_bert_base_fc2_full_size_twelve_layers(path, monkeypatch):
     if path == "stream":
         monkeypatch.setenv("ZIPLM_NEURON_PATH", "stream")
-    elif path == "lazy_tc":
-        monkeypatch.setenv("ZIPLM_LAZY_UPDATE", "tc")
     shape = wl.CONFIGS["c3_bert_base_fc2"][0]
     checked = [0, 7]
     W, H_or, out = run_full(shape, checked)

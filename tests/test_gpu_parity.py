@@ -195,17 +195,13 @@ def test_not_positive_definite_layer_is_flagged_and_others_finish():
 
 
 # ------------------------------------------------------------------ neuron path (a4 - a10)
-@pytest.fixture(params=["lazy", "lazy_tc", "stream"])
+@pytest.fixture(params=["lazy", "stream"])
 def neuron_path(request, monkeypatch):
     """Run a test once per neuron-path variant: delayed rank-B updates (default where the shape
-    allows it), the same with the tcgen05 variant of the rank-B update of H^-1 and Q, and the
-    per-step streaming update."""
+    allows it) and the per-step streaming update."""
     monkeypatch.delenv("ZIPLM_NEURON_PATH", raising=False)
-    monkeypatch.delenv("ZIPLM_LAZY_UPDATE", raising=False)
     if request.param == "stream":
         monkeypatch.setenv("ZIPLM_NEURON_PATH", "stream")
-    elif request.param == "lazy_tc":
-        monkeypatch.setenv("ZIPLM_LAZY_UPDATE", "tc")
     return request.param
 
 
