@@ -366,7 +366,7 @@ def run_ours(args, shape):
     # ---- one more step with per-phase event timing (roofline of the dominant kernel), and one
     # with the per-step streaming update selected, whose fused H^-1 / W kernel is reported too
     # (layer groups are run back to back here, so that a kernel's time is its own)
-    os.environ["ZIPLM_LAYER_GROUPS"] = "1"
+    z.set_option(z.Option.LAYER_GROUPS, 1)
     step()
     torch.cuda.synchronize()
     e0.record()
@@ -380,14 +380,14 @@ def run_ours(args, shape):
     phases = z.profile_end()
     phases_stream = {"update": (0.0, 0)}
     if not args.skip_stream_leg:
-        os.environ["ZIPLM_NEURON_PATH"] = "stream"
+        z.set_option(z.Option.NEURON_PATH, 1)
         step()
         z.profile_begin()
         step()
         torch.cuda.synchronize()
         phases_stream = z.profile_end()
-        del os.environ["ZIPLM_NEURON_PATH"]
-    del os.environ["ZIPLM_LAYER_GROUPS"]
+        z.set_option(z.Option.NEURON_PATH, 0)
+    z.set_option(z.Option.LAYER_GROUPS, 0)
 
     # ---- the Hessian from token-major activations (one token per row, the layout a forward pass
     # emits): one call on the whole calibration set, and eight calibration batches with beta = 1
@@ -596,7 +596,7 @@ def run_ours(args, shape):
                 traffic_note=NCU_TRAFFIC["k_neuron_update"], peak_source=peak_src, launches=upd_n,
                 avg_launch_us=1e3 * upd_ms / max(upd_n, 1), algorithmic_bytes_per_step=alg_bytes,
                 note="per-step fused H^-1/W update of the streaming variant "
-                     "(ZIPLM_NEURON_PATH=stream), timed in a separate step",
+                     "(option NEURON_PATH = 1), timed in a separate step",
                 phases_ms={k: round(v[0], 3) for k, v in phases_stream.items() if v[1] > 0}),
         )
         if tok is not None:

@@ -6,7 +6,9 @@
  *   - "dev" pointers are CUDA device pointers of the current device, "host" pointers are
  *     ordinary host memory.  All matrices are dense row-major.
  *   - The caller owns every buffer.  The library allocates no device memory and keeps no state
- *     between calls (the optional diagnostics at the end of this file aside).
+ *     between calls, apart from the diagnostics at the end of this file, the stream pool of
+ *     ziplm_prune_layers described next and the built-in scratch of
+ *     ziplm_damped_inverse_noalloc.  Calls may be made from several host threads.
  *   - All work is ordered on `cuda_stream` (a cudaStream_t passed as void*, NULL = the default
  *     stream) and the call returns without synchronising: it starts after everything already
  *     enqueued there and the stream continues only when it is complete.  Buffers must stay alive
@@ -72,6 +74,10 @@ const char* ziplm_status_string(ziplm_status s);
  * Errors: ZIPLM_ERR_INVALID_ARG for L, d < 1, n_tokens < 0, ldx < n_tokens, a NULL pointer,
  * misaligned X or beta outside {0, 1}; ZIPLM_ERR_WORKSPACE; ZIPLM_ERR_CUDA.
  * n_tokens = 0 scales H by beta and returns.
+ * Every wait inside the tensor-core kernel is bounded.  Should one run out (it cannot on a healthy
+ * device), the call has no status output of its own: H[l][0][0] of every layer is NaN on return,
+ * so that ziplm_damped_inverse or ziplm_prune_layers on that H reports ZIPLM_ERR_NONFINITE for
+ * every layer.  The same holds for ziplm_hessian_accumulate_tokens.
  */
 size_t ziplm_hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype x_dtype);
 
@@ -180,7 +186,8 @@ ziplm_status ziplm_damped_inverse_noalloc(const float* H, int L, int d, float da
  * the reconstruction loss of Eq. 1.
  *
  *   W            dev, [L, d_row, d_col] fp32; not modified
- *   H            dev, [L, d_col, d_col] fp32, the UNDAMPED 2 X X^T, symmetric; not modified
+ *   H            dev, [L, d_col, d_col] fp32, the UNDAMPED 2 X X^T, symmetric; not modified;
+ *                16-byte aligned (ZIPLM_ERR_INVALID_ARG otherwise)
  *   group_size   columns per structure; d_col % group_size == 0; 1 <= group_size <= 64
  *   damp_frac    lambda = damp_frac * mean(diag H[l]); >= 0
  *   levels       HOST, [n_levels] numbers of REMAINING structures, strictly decreasing, each in
@@ -340,8 +347,26 @@ ziplm_status ziplm_search_levels(const float* loss, const float* base_loss, cons
                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
- * Diagnostics (no counterpart in the paper): a launch counter and optional per-phase timing.
+ * Diagnostics (no counterpart in the paper): options, a launch counter and optional per-phase
+ * timing.  This is the only process-wide state the library keeps besides an internal pool of
+ * streams (see ziplm_prune_layers); no environment variable is read.
  *
+ * ziplm_set_option         sets a process-wide option that later calls read when they start; every
+ *                          option defaults to 0.  ZIPLM_ERR_INVALID_ARG for an unknown option or a
+ *                          value outside its range.  Results never depend on an option beyond
+ *                          rounding (every variant passes the same parity tests).
+ *     ZIPLM_OPT_NEURON_PATH       0: delayed rank-32 updates where the shape allows them
+ *                                 (d_col % 4 == 0, d_col <= 6144); 1: per-step streaming update.
+ *     ZIPLM_OPT_LAYER_GROUPS      0: default (6); 1..8: number of layer groups that
+ *                                 ziplm_prune_layers runs on internal streams (1 = none).
+ *     ZIPLM_OPT_FORCE_BLOCK_PATH  1: group_size 1 takes the general block path (float64 state).
+ *                                 The only option ziplm_prune_workspace_bytes depends on: set it
+ *                                 before the query and leave it until the call.
+ *     ZIPLM_OPT_HESSIAN_ROUTE     0: tensor cores from 32 tokens on; 1: CUDA-core kernel always.
+ *     ZIPLM_OPT_SPIN_LIMIT        0: default; n > 0: poll limit of the Hessian kernel's wait for a
+ *                                 free pipeline stage (tests make a bounded wait run out with it;
+ *                                 see ziplm_hessian_accumulate for how that is reported).
+ * ziplm_get_option         current value of an option.
  * ziplm_launch_count       kernels launched by this library since it was loaded.
  * ziplm_profile_begin      from now on every phase of every call is bracketed by a pair of CUDA
  *                          events on the caller's stream (process-wide switch, not re-entrant;
@@ -352,6 +377,16 @@ ziplm_status ziplm_search_levels(const float* loss, const float* base_loss, cons
  * ziplm_profile_phase_count / ziplm_profile_phase_name   enumerate the phases ("hessian",
  *                          "inverse", "init", "prep", "update", "snapshot", "lazy_steps", ...).
  */
+typedef enum {
+    ZIPLM_OPT_NEURON_PATH = 0,
+    ZIPLM_OPT_LAYER_GROUPS = 1,
+    ZIPLM_OPT_FORCE_BLOCK_PATH = 2,
+    ZIPLM_OPT_HESSIAN_ROUTE = 3,
+    ZIPLM_OPT_SPIN_LIMIT = 4,
+    ZIPLM_OPT_COUNT = 5
+} ziplm_option;
+ziplm_status ziplm_set_option(ziplm_option option, int value);
+int ziplm_get_option(ziplm_option option);
 long long ziplm_launch_count(void);
 ziplm_status ziplm_profile_begin(void);
 ziplm_status ziplm_profile_end(double* phase_ms, long long* phase_spans, int n_phases);

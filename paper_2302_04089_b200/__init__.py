@@ -9,5 +9,5 @@ from .binding import (  # noqa: F401
     hessian_tokens_workspace_bytes, damped_inverse, damped_inverse_noalloc, prune_layers,
     status_string, hessian_workspace_bytes, inverse_workspace_bytes, prune_workspace_bytes,
     kept_structures, gather_columns, gather_rows, select_levels, select_workspace_bytes,
-    search_levels, search_workspace_bytes, launch_count, profile_begin, profile_end, profile_phase_count, profile_phase_name,
+    search_levels, search_workspace_bytes, Option, set_option, get_option, launch_count, profile_begin, profile_end, profile_phase_count, profile_phase_name,
 )

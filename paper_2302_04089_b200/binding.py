@@ -95,6 +95,10 @@ def load_library() -> ctypes.CDLL:
     lib.ziplm_search_levels.restype = c_int
     lib.ziplm_search_levels.argtypes = [vp, vp, vp, vp, c_int, c_int, vp, vp, vp, c_int, c_int, vp, vp,
                                         c_int, vp, vp, vp, vp, vp, vp, c_sz, vp]
+    lib.ziplm_set_option.restype = c_int
+    lib.ziplm_set_option.argtypes = [c_int, c_int]
+    lib.ziplm_get_option.restype = c_int
+    lib.ziplm_get_option.argtypes = [c_int]
     lib.ziplm_launch_count.restype = ctypes.c_longlong
     lib.ziplm_launch_count.argtypes = []
     lib.ziplm_profile_begin.restype = c_int
@@ -435,6 +439,25 @@ def search_levels(loss: torch.Tensor, base_loss: torch.Tensor, time: torch.Tenso
     if st != 0:
         raise ZiplmError(st, "ziplm_search_levels")
     return out
+
+
+class Option:
+    """Diagnostic options of ziplm_set_option (all default to 0)."""
+    NEURON_PATH = 0          # 1: per-step streaming update instead of delayed rank-32 updates
+    LAYER_GROUPS = 1         # 1..8 layer groups on internal streams (0: default)
+    FORCE_BLOCK_PATH = 2     # 1: group_size 1 through the general block path
+    HESSIAN_ROUTE = 3        # 1: CUDA-core Hessian kernel always
+    SPIN_LIMIT = 4           # poll limit of the Hessian kernel's wait for a free pipeline stage
+
+
+def set_option(option: int, value: int) -> None:
+    st = load_library().ziplm_set_option(int(option), int(value))
+    if st != 0:
+        raise ZiplmError(st, "ziplm_set_option")
+
+
+def get_option(option: int) -> int:
+    return int(load_library().ziplm_get_option(int(option)))
 
 
 def launch_count() -> int:

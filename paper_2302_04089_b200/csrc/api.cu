@@ -1,7 +1,6 @@
 // extern "C" boundary: argument validation and dispatch.  No device memory is allocated here and
 // nothing synchronises; every stage is enqueued on the caller's stream.
 #include <math.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -11,12 +10,9 @@ namespace {
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-// Debugging switch: ZIPLM_FORCE_BLOCK_PATH=1 sends group_size 1 through the general block path
-// (float64 state, g x g Cholesky per structure) instead of the streaming neuron path.
-bool force_block_path() {
-    const char* e = getenv("ZIPLM_FORCE_BLOCK_PATH");
-    return e && e[0] == '1';
-}
+// Diagnostic option: group_size 1 goes through the general block path (float64 state, g x g
+// Cholesky per structure) instead of the neuron path.
+bool force_block_path() { return option_value(ZIPLM_OPT_FORCE_BLOCK_PATH) == 1; }
 
 bool have_device() {
     int dev = -1;
@@ -124,6 +120,7 @@ ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row
     if (L < 1 || d_row < 1 || d_col < 1 || group_size < 1 || n_levels < 0) return ZIPLM_ERR_INVALID_ARG;
     if (d_col % group_size != 0) return ZIPLM_ERR_INVALID_ARG;
     if (!W || !H || !order || !layer_status) return ZIPLM_ERR_INVALID_ARG;
+    if (!aligned(H, 16)) return ZIPLM_ERR_INVALID_ARG;      // H is read with 128-bit loads
     if (n_levels > 0 && (!levels || !W_snap || !loss)) return ZIPLM_ERR_INVALID_ARG;
     if (!(damp_frac >= 0.f) || !isfinite(damp_frac)) return ZIPLM_ERR_INVALID_ARG;
     const int G = d_col / group_size;

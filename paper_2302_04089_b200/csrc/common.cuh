@@ -32,6 +32,9 @@ struct Carver {
 // Number of kernels launched by this library since it was loaded (diagnostics).
 extern std::atomic<long long> g_launches;
 
+// Current value of a diagnostic option (ziplm_set_option); 0 is every option's default.
+int option_value(int option);
+
 // Phases reported by the optional event timing (ziplm_profile_begin / ziplm_profile_end).
 enum Phase { PH_HESSIAN = 0, PH_INVERSE, PH_INIT, PH_PREP, PH_UPDATE, PH_SNAPSHOT, PH_BLOCK_SCORE,
              PH_BLOCK_UPDATE, PH_LAZY_STEPS, PH_LAZY_UPDATE_AQ, PH_LAZY_UPDATE_W, PH_INV_PRODUCTS,

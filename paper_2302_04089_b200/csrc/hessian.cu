@@ -7,11 +7,9 @@
 // two-level fp32 sum (the running tile sum is folded into a second accumulator every 512 tokens,
 // which keeps the rounding error of a 1e4 .. 1e5 term sum near the fp32 unit roundoff).  The
 // tensor-core route (hessian_tc.cu) is the default; the CUDA-core route serves token counts
-// below one K block and can be forced with ZIPLM_HESSIAN_ROUTE=simt for comparison.
+// below one K block and can be forced with ziplm_set_option(ZIPLM_OPT_HESSIAN_ROUTE, 1) for comparison.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
-#include <stdlib.h>
-#include <string.h>
 
 #include "common.cuh"
 
@@ -139,16 +137,15 @@ __global__ void k_scale_h(float* __restrict__ H, size_t count, float beta) {
 }
 
 bool use_tensor_cores(long long N) {
-    const char* e = getenv("ZIPLM_HESSIAN_ROUTE");
-    if (e && strcmp(e, "simt") == 0) return false;
-    if (e && strcmp(e, "tc") == 0) return N > 0;
+    if (option_value(ZIPLM_OPT_HESSIAN_ROUTE) == 1) return false;   // CUDA-core kernel
     return N >= 32;
 }
 
 }  // namespace
 
 size_t hessian_workspace_bytes(int L, int d, long long n_tokens, ziplm_dtype dt, bool token_major) {
-    return use_tensor_cores(n_tokens) ? hessian_tc_workspace_bytes(L, d, n_tokens, dt, token_major) : 0;
+    // the larger of the two routes' needs, whatever route the call will take
+    return n_tokens > 0 ? hessian_tc_workspace_bytes(L, d, n_tokens, dt, token_major) : 0;
 }
 
 ziplm_status run_hessian(float* H, const void* X, ziplm_dtype dt, bool token_major, int L, int d,

@@ -14,9 +14,11 @@
 //
 // One CTA per tile: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..9 =
 // epilogue (two per TMEM lane quarter; they drain the accumulator every few K blocks, see
-// below).  Every mbarrier wait is bounded; if one runs out the
-// kernel raises the error word, poisons H[l][0][0] with NaN and leaves through the normal exit
-// (TMEM freed), so a lost copy can never hang the GPU.
+// below).  Every mbarrier wait is bounded; if one runs out the kernel raises the error word and
+// every role leaves its loop; the issuer then waits (one more commit) for the MMAs it has issued,
+// the producer for the copies it has started, and the CTA leaves through the normal exit (TMEM
+// freed), so a lost copy can never hang the GPU.  A small kernel after the product launches turns
+// a raised error word into NaN in H[l][0][0] of every layer.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -52,12 +54,12 @@ template <bool TF32>
 __global__ void __launch_bounds__(THREADS, 1)
 k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
           float* __restrict__ H, int d, int num_kb, float alpha, float beta, int layer0,
-          int* __restrict__ err_word, uint32_t fmt16) {
+          int* __restrict__ err_word, uint32_t fmt16, uint32_t empty_spin_limit) {
     using C = Cfg<TF32>;
     constexpr int STAGE_BYTES = C::TILES * TILE_BYTES;
     constexpr uint32_t TMEM_COLS = TF32 ? 512u : 256u;   // main x2 (+ cross terms), power of two
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bar_full[C::STAGES], bar_empty[C::STAGES], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint64_t bar_full[C::STAGES], bar_empty[C::STAGES], bar_acc_full[2], bar_acc_empty[2], bar_final;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -82,6 +84,7 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
             mbar_init(smem_u32(&bar_acc_full[b]), 1);
             mbar_init(smem_u32(&bar_acc_empty[b]), EPI_WARPS);   // one arrival per epilogue warp
         }
+        mbar_init(smem_u32(&bar_final), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -95,6 +98,7 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
     const uint32_t tmem_base = tmem_base_slot;            // main[0] = +0, main[1] = +128, cross = +256
     volatile int* abortp = &abort_flag;
     bool failed = false;
+    int issued = 0;                                       // K blocks whose copies were started (thread 0)
 
     if (warp == 0) {
         if (lane == 0) {
@@ -103,7 +107,10 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
             for (int kb = 0; kb < num_kb; ++kb) {
                 const int s = kb % C::STAGES;
                 const uint32_t ph = (uint32_t)(kb / C::STAGES) & 1u;
-                if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, abortp)) { failed = true; break; }
+                if (!mbar_wait_limit(smem_u32(&bar_empty[s]), ph ^ 1u, abortp, empty_spin_limit)) {
+                    failed = true;
+                    break;
+                }
                 const uint32_t full = smem_u32(&bar_full[s]);
                 const uint32_t base = tiles + (uint32_t)s * STAGE_BYTES;
                 mbar_expect_tx(full, bytes);
@@ -114,6 +121,7 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
                     tma_load_3d(base + 2 * TILE_BYTES, &map_lo, full, x, i0, l);
                     if (!diag) tma_load_3d(base + 3 * TILE_BYTES, &map_lo, full, x, j0, l);
                 }
+                issued = kb + 1;
             }
         }
     } else if (warp == 1) {
@@ -160,6 +168,10 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
                 }
                 if (!failed) umma_commit(smem_u32(&bar_acc_full[b]));   // chunk (and all before) done
             }
+            // Whatever was issued has completed before tensor memory is given back and the CTA
+            // retires, also when a role has given up: one more commit, to a barrier of its own.
+            umma_commit(smem_u32(&bar_final));
+            mbar_wait_quiet(smem_u32(&bar_final), 0u);
         }
     } else {
         // ---------------- epilogue: warps 2..9; TMEM lane quarter = warp % 4, column half by warp
@@ -224,20 +236,25 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (abort_flag) {
-        // give copies that are still in flight a bounded chance to land before the CTA retires
-        if (threadIdx.x == 0) {
-            for (int s = 0; s < C::STAGES; ++s)
-                for (uint32_t it = 0; it < 4096u; ++it)
-                    if (mbar_try_wait(smem_u32(&bar_full[s]), 0u) || mbar_try_wait(smem_u32(&bar_full[s]), 1u))
-                        break;
-            H[(size_t)(layer0 + l) * d * d] = __int_as_float(0x7fc00000);
-        }
+        // Copies that were started land in this CTA's shared memory: wait for them (bounded) before
+        // the CTA retires.  The last STAGES K blocks started are the latest phases of their barriers.
+        if (threadIdx.x == 0)
+            for (int kb = issued > C::STAGES ? issued - C::STAGES : 0; kb < issued; ++kb)
+                mbar_wait_quiet(smem_u32(&bar_full[kb % C::STAGES]), (uint32_t)(kb / C::STAGES) & 1u);
         __syncthreads();
     }
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
                      : "memory");
     }
+}
+
+// A product kernel that gave up on a wait leaves ZIPLM_ERR_TIMEOUT in the error word; the layers'
+// first entries then become NaN, after every product launch of the call, so that whichever stage
+// reads H next reports ZIPLM_ERR_NONFINITE.
+__global__ void k_hessian_flag_timeout(float* __restrict__ H, int L, int d, const int* __restrict__ err_word) {
+    const int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l < L && *err_word != 0) H[(size_t)l * d * d] = __int_as_float(0x7fc00000);
 }
 
 // X_hi = X with the 13 low mantissa bits cleared (exactly a TF32 value), X_lo = X - X_hi (exact).
@@ -430,6 +447,8 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
     Carver c(ws);
     int* err_word = c.take<int>(1);
     ZIPLM_CHECK_CUDA(cudaMemsetAsync(err_word, 0, sizeof(int), st));
+    const int spin_opt = option_value(ZIPLM_OPT_SPIN_LIMIT);
+    const uint32_t spin = spin_opt > 0 ? (uint32_t)spin_opt : kSpinLimit;
     const int T = (d + TM - 1) / TM;
     const int n_tiles = T * (T + 1) / 2;
     const size_t smem_tf32 = (size_t)Cfg<true>::STAGES * Cfg<true>::TILES * TILE_BYTES + 1024;
@@ -481,7 +500,7 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
             if (!make_map(&mh, hi, ZIPLM_F32, N, d, ln, np) || !make_map(&ml, lo, ZIPLM_F32, N, d, ln, np))
                 return ZIPLM_ERR_CUDA;
             k_syrk_tc<true><<<dim3(n_tiles, ln), THREADS, smem_tf32, st>>>(mh, ml, H, d, num_kb, alpha, beta,
-                                                                      l0, err_word, 2u);
+                                                                      l0, err_word, 2u, spin);
             ZIPLM_CHECK_LAUNCH();
         }
     } else if (token_major) {
@@ -505,7 +524,7 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
             CUtensorMap mx;
             if (!make_map(&mx, xt, dt, N, d, ln, np)) return ZIPLM_ERR_CUDA;
             k_syrk_tc<false><<<dim3(n_tiles, ln), THREADS, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
-                                                                       l0, err_word, fmt16);
+                                                                       l0, err_word, fmt16, spin);
             ZIPLM_CHECK_LAUNCH();
         }
     } else {
@@ -518,10 +537,12 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
             const __nv_bfloat16* Xc = static_cast<const __nv_bfloat16*>(X) + (size_t)l0 * d * ldx;
             if (!make_map(&mx, Xc, dt, N, d, ln, ldx)) return ZIPLM_ERR_CUDA;
             k_syrk_tc<false><<<dim3(n_tiles, ln), THREADS, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
-                                                                       l0, err_word, fmt16);
+                                                                       l0, err_word, fmt16, spin);
             ZIPLM_CHECK_LAUNCH();
         }
     }
+    k_hessian_flag_timeout<<<(L + 127) / 128, 128, 0, st>>>(H, L, d, err_word);
+    ZIPLM_CHECK_LAUNCH();
     return ZIPLM_OK;
 }
 

@@ -718,7 +718,7 @@ int task_ctas(const GemmTask& t) {
 
 ziplm_status launch_pair(const InvCtx& c, const GemmTask& t1, const GemmTask& t2) {
     const int n1 = task_ctas(t1), n2 = task_ctas(t2);
-    static const cudaError_t attr = cudaFuncSetAttribute(
+    const cudaError_t attr = cudaFuncSetAttribute(
         k_dgemm_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
     if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
     PhaseScope ps(PH_INV_PRODUCTS, c.st);
@@ -731,7 +731,7 @@ template <bool TA, bool TB>
 ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
     const int ctas = task_ctas(t);
     if (ctas <= 0 || t.kt <= 0) return ZIPLM_OK;
-    static const cudaError_t attr = cudaFuncSetAttribute(
+    const cudaError_t attr = cudaFuncSetAttribute(
         k_dgemm_tiles<TA, TB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
     if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
     PhaseScope ps(PH_INV_PRODUCTS, c.st);
@@ -744,7 +744,7 @@ ziplm_status launch_gemm(const InvCtx& c, const GemmTask& t) {
 // and M its inverse.
 ziplm_status factor_range(const InvCtx& c, int lo, int hi) {
     if (hi - lo <= kSmallMax) {
-        static const cudaError_t attr = cudaFuncSetAttribute(
+        const cudaError_t attr = cudaFuncSetAttribute(
             k_factor_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmallSmem));
         if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
         PhaseScope ps(PH_INV_LEAVES, c.st);
@@ -824,7 +824,7 @@ ziplm_status run_damped_inverse(const float* H, int L, int d, float damp_frac, d
     if (s != ZIPLM_OK) return s;
     {
         PhaseScope ps(PH_INV_LAUUM, st);
-        static const cudaError_t attr = cudaFuncSetAttribute(
+        const cudaError_t attr = cudaFuncSetAttribute(
             k_lauum, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProductSmemBytes);
         if (attr != cudaSuccess) return ZIPLM_ERR_CUDA;
         k_lauum<<<dim3(lower_macro_count(T), L), GT, kProductSmemBytes, st>>>(ctx.M, dp, T, d, out64, tri32,

@@ -11,6 +11,12 @@ namespace ziplm {
 
 std::atomic<long long> g_launches{0};
 
+static std::atomic<int> g_options[ZIPLM_OPT_COUNT];
+
+int option_value(int option) {
+    return (option >= 0 && option < ZIPLM_OPT_COUNT) ? g_options[option].load(std::memory_order_relaxed) : 0;
+}
+
 namespace {
 struct Span { int phase; cudaEvent_t a, b; };
 std::mutex g_mu;
@@ -47,6 +53,18 @@ using namespace ziplm;
 extern "C" {
 
 long long ziplm_launch_count(void) { return g_launches.load(); }
+
+ziplm_status ziplm_set_option(ziplm_option option, int value) {
+    if (option < 0 || option >= ZIPLM_OPT_COUNT || value < 0) return ZIPLM_ERR_INVALID_ARG;
+    if ((option == ZIPLM_OPT_NEURON_PATH || option == ZIPLM_OPT_FORCE_BLOCK_PATH ||
+         option == ZIPLM_OPT_HESSIAN_ROUTE) && value > 1)
+        return ZIPLM_ERR_INVALID_ARG;
+    if (option == ZIPLM_OPT_LAYER_GROUPS && value > 8) return ZIPLM_ERR_INVALID_ARG;
+    ziplm::g_options[option].store(value, std::memory_order_relaxed);
+    return ZIPLM_OK;
+}
+
+int ziplm_get_option(ziplm_option option) { return ziplm::option_value((int)option); }
 
 int ziplm_profile_phase_count(void) { return PH_COUNT; }
 

@@ -28,7 +28,6 @@
 #include <cooperative_groups.h>
 #include <math.h>
 
-#include <stdlib.h>
 
 #include "common.cuh"
 

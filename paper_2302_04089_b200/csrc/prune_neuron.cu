@@ -23,8 +23,9 @@
 // Algorithm 1 -- so they are simply dropped).  The live problem is therefore always the leading
 // n x n corner, and every step streams exactly the live bytes.
 #include <math.h>
-#include <stdlib.h>
-#include <string.h>
+
+#include <mutex>
+#include <vector>
 
 #include "common.cuh"
 
@@ -377,10 +378,9 @@ NeuronWs carve_neuron(void* ws, int L, int r, int d) {
 }  // namespace
 
 // The delayed-update variant (prune_lazy.cu) is the default where it applies; the streaming
-// variant in this file serves the other shapes and ZIPLM_NEURON_PATH=stream selects it always.
+// variant in this file serves the other shapes and ziplm_set_option(ZIPLM_OPT_NEURON_PATH, 1) selects it always.
 static bool use_lazy_path(int d) {
-    const char* e = getenv("ZIPLM_NEURON_PATH");
-    if (e && strcmp(e, "stream") == 0) return false;
+    if (option_value(ZIPLM_OPT_NEURON_PATH) == 1) return false;
     return lazy_path_supported(d);
 }
 
@@ -392,10 +392,8 @@ constexpr int kMaxGroups = 8;
 constexpr int kDefaultGroups = 6;
 
 static int layer_groups(int L) {
-    int g = kDefaultGroups;
-    const char* e = getenv("ZIPLM_LAYER_GROUPS");
-    if (e) g = atoi(e);
-    if (g < 1) g = 1;
+    int g = option_value(ZIPLM_OPT_LAYER_GROUPS);
+    if (g < 1) g = kDefaultGroups;
     if (g > kMaxGroups) g = kMaxGroups;
     if (g > L) g = L;
     return g;
@@ -411,19 +409,66 @@ static size_t grouped_lazy_bytes(int L, int r, int d, int n_levels, int groups) 
     return b;
 }
 
-// Internal streams, created once per device and kept for the life of the process.
-static cudaStream_t* group_streams() {
-    static cudaStream_t pool[64][kMaxGroups] = {};
-    static bool ready[64] = {};
+// Internal streams and the fork / join events of a call, created once per device and kept for
+// the life of the process.  Several host threads may call at the same time: the pool is built
+// under a mutex, and every call takes an event set of its own from a free list (a set can be
+// used again as soon as the call that held it has enqueued its work, since a stream wait refers
+// to the record that precedes it).
+struct EventSet {
+    cudaEvent_t fork;
+    cudaEvent_t join[kMaxGroups];
+};
+struct DevicePool {
+    bool ready = false;
+    cudaStream_t streams[kMaxGroups] = {};
+    std::vector<EventSet*> free_sets;
+};
+static std::mutex g_pool_mu;
+static DevicePool g_pools[64];
+
+static DevicePool* device_pool() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!ready[dev]) {
+    std::lock_guard<std::mutex> lk(g_pool_mu);
+    DevicePool& p = g_pools[dev];
+    if (!p.ready) {
         for (int g = 0; g < kMaxGroups; ++g)
-            if (cudaStreamCreateWithFlags(&pool[dev][g], cudaStreamNonBlocking) != cudaSuccess)
+            if (cudaStreamCreateWithFlags(&p.streams[g], cudaStreamNonBlocking) != cudaSuccess) {
+                for (int h = 0; h < g; ++h) cudaStreamDestroy(p.streams[h]);
                 return nullptr;
-        ready[dev] = true;
+            }
+        p.ready = true;
     }
-    return pool[dev];
+    return &p;
+}
+
+static EventSet* take_events(DevicePool* p) {
+    {
+        std::lock_guard<std::mutex> lk(g_pool_mu);
+        if (!p->free_sets.empty()) {
+            EventSet* e = p->free_sets.back();
+            p->free_sets.pop_back();
+            return e;
+        }
+    }
+    EventSet* e = new EventSet();
+    const bool fork_ok = cudaEventCreateWithFlags(&e->fork, cudaEventDisableTiming) == cudaSuccess;
+    int made = 0;
+    while (fork_ok && made < kMaxGroups &&
+           cudaEventCreateWithFlags(&e->join[made], cudaEventDisableTiming) == cudaSuccess)
+        ++made;
+    if (made < kMaxGroups) {             // give back what was created
+        for (int g = 0; g < made; ++g) cudaEventDestroy(e->join[g]);
+        if (fork_ok) cudaEventDestroy(e->fork);
+        delete e;
+        return nullptr;
+    }
+    return e;
+}
+
+static void give_events(DevicePool* p, EventSet* e) {
+    std::lock_guard<std::mutex> lk(g_pool_mu);
+    p->free_sets.push_back(e);
 }
 
 size_t neuron_workspace_bytes(int L, int r, int d, int n_levels) {
@@ -443,8 +488,9 @@ static ziplm_status run_prune_lazy_grouped(const float* W, const float* H, int L
                                            float* saliency, int* layer_status, void* ws,
                                            cudaStream_t st) {
     const int groups = layer_groups(L);
-    cudaStream_t* pool = groups > 1 ? group_streams() : nullptr;
-    if (groups <= 1 || !pool)
+    DevicePool* pool = groups > 1 ? device_pool() : nullptr;
+    EventSet* ev = pool ? take_events(pool) : nullptr;
+    if (groups <= 1 || !ev)
         return run_prune_lazy(W, H, L, r, d, damp_frac, levels, n_levels, W_snap, loss, base_loss,
                               order, saliency, layer_status, ws,
                               lazy_workspace_bytes(L, r, d, n_levels), st);
@@ -452,16 +498,17 @@ static ziplm_status run_prune_lazy_grouped(const float* W, const float* H, int L
     // concurrently (different layers on different streams) do not queue behind each other.
     static std::atomic<unsigned> next_stream{0};
     const unsigned first = next_stream.fetch_add((unsigned)groups);
-    cudaEvent_t fork, join[kMaxGroups];
-    ZIPLM_CHECK_CUDA(cudaEventCreateWithFlags(&fork, cudaEventDisableTiming));
-    ZIPLM_CHECK_CUDA(cudaEventRecord(fork, st));
+    if (cudaEventRecord(ev->fork, st) != cudaSuccess) {
+        give_events(pool, ev);
+        return ZIPLM_ERR_CUDA;
+    }
     ziplm_status rc = ZIPLM_OK;
     char* wsp = static_cast<char*>(ws);
     for (int g = 0; g < groups; ++g) {
         const int l0 = group_begin(L, groups, g), Lg = group_begin(L, groups, g + 1) - l0;
         const size_t bytes = lazy_workspace_bytes(Lg, r, d, n_levels);
-        cudaStream_t sg = pool[(first + (unsigned)g) % kMaxGroups];
-        bool ok = cudaStreamWaitEvent(sg, fork, 0) == cudaSuccess;
+        cudaStream_t sg = pool->streams[(first + (unsigned)g) % kMaxGroups];
+        bool ok = cudaStreamWaitEvent(sg, ev->fork, 0) == cudaSuccess;
         if (ok && rc == ZIPLM_OK)
             rc = run_prune_lazy(W + (size_t)l0 * r * d, H + (size_t)l0 * d * d, Lg, r, d, damp_frac,
                                 levels, n_levels, W_snap + (size_t)l0 * n_levels * r * d,
@@ -469,16 +516,12 @@ static ziplm_status run_prune_lazy_grouped(const float* W, const float* H, int L
                                 order + (size_t)l0 * d, saliency ? saliency + (size_t)l0 * d : nullptr,
                                 layer_status + l0, wsp, bytes, sg);
         // always join, so that the caller's stream stays ordered after whatever was enqueued
-        ok = ok && cudaEventCreateWithFlags(&join[g], cudaEventDisableTiming) == cudaSuccess;
-        if (ok) {
-            ok = cudaEventRecord(join[g], sg) == cudaSuccess &&
-                 cudaStreamWaitEvent(st, join[g], 0) == cudaSuccess;
-            cudaEventDestroy(join[g]);
-        }
+        ok = ok && cudaEventRecord(ev->join[g], sg) == cudaSuccess &&
+             cudaStreamWaitEvent(st, ev->join[g], 0) == cudaSuccess;
         if (!ok && rc == ZIPLM_OK) rc = ZIPLM_ERR_CUDA;
         wsp += bytes;
     }
-    cudaEventDestroy(fork);
+    give_events(pool, ev);
     return rc;
 }
 

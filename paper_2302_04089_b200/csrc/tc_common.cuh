@@ -40,6 +40,37 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return false;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait with a caller-given poll limit.  The default limit takes the ordinary wait; a
+// smaller one polls without ever suspending the thread, so that a limit of 1 is exactly one look
+// at the barrier.
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                uint32_t limit) {
+    if (limit >= kSpinLimit) return mbar_wait(bar, parity, abort_flag);
+    for (uint32_t it = 0; it < limit; ++it) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u && *abort_flag) return false;
+    }
+    return false;
+}
+// Bounded wait that does not look at the abort flag: used on the way out of a kernel, for work
+// that has already been issued and will complete.
+__device__ __forceinline__ bool mbar_wait_quiet(uint32_t bar, uint32_t parity) {
+    const long long t0 = clock64();
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u && clock64() - t0 > kSpinClocks) return false;
+    }
+    return false;
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int x, int y, int z) {
     asm volatile(

@@ -55,6 +55,36 @@ def test_status_strings_and_workspace_queries(lib):
     assert lib.ziplm_select_workspace_bytes(0, 24, 10000) == 0
 
 
+def test_options_round_trip_and_reject_bad_values(lib):
+    lib.ziplm_set_option.restype = ctypes.c_int
+    lib.ziplm_get_option.restype = ctypes.c_int
+    for opt, good, bad in ((0, 1, 2), (1, 8, 9), (2, 1, 2), (3, 1, 5), (4, 1000, -1)):
+        assert lib.ziplm_get_option(opt) == 0
+        assert lib.ziplm_set_option(opt, good) == 0 and lib.ziplm_get_option(opt) == good
+        assert lib.ziplm_set_option(opt, bad) == 1 and lib.ziplm_get_option(opt) == good
+        assert lib.ziplm_set_option(opt, 0) == 0
+    assert lib.ziplm_set_option(5, 0) == 1 and lib.ziplm_set_option(-1, 0) == 1
+    assert lib.ziplm_get_option(17) == 0
+
+
+def test_prune_layers_rejects_a_misaligned_hessian_on_the_host(lib):
+    """H is read with 128-bit loads: a pointer that is not 16-byte aligned is refused before
+    anything is enqueued (only the return code is looked at; nothing is launched)."""
+    lib.ziplm_prune_layers.restype = ctypes.c_int
+    lib.ziplm_prune_layers.argtypes = [ctypes.c_void_p] * 2 + [ctypes.c_int] * 4 + [ctypes.c_float] + \
+        [ctypes.c_void_p, ctypes.c_int] + [ctypes.c_void_p] * 7 + [ctypes.c_size_t, ctypes.c_void_p]
+    levels = (ctypes.c_int * 1)(4)
+    base = 1 << 20                       # never dereferenced: the call stops at the argument checks
+
+    def call(h_addr):
+        return lib.ziplm_prune_layers(base, h_addr, 1, 8, 8, 1, 0.01, levels, 1, base, base, None,
+                                      base, None, base, None, 0, None)
+
+    assert call(base + 4096 + 4) == 1            # ZIPLM_ERR_INVALID_ARG
+    assert call(base + 4096 + 8) == 1
+    assert call(base + 4096) == 2                # aligned: next check is the (missing) workspace
+
+
 def test_binding_mirrors_the_abi_names():
     import paper_2302_04089_b200 as z
     for name in declared_symbols():

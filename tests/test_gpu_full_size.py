@@ -53,6 +53,18 @@ def run_full(shape, check_layers):
     return W, H_or, out
 
 
+@pytest.fixture
+def neuron_variant():
+    """Selects the neuron-path variant for one test and restores the default afterwards."""
+    z = zb()
+
+    def choose(path):
+        z.set_option(z.Option.NEURON_PATH, 1 if path == "stream" else 0)
+
+    yield choose
+    z.set_option(z.Option.NEURON_PATH, 0)
+
+
 def generic_properties(shape, out):
     G, L = shape.n_groups, shape.n_layers
     levels = list(shape.levels)
@@ -128,9 +140,8 @@ def lockstep_head(W, H32, shape, out, layer, n_steps):
 
 
 @pytest.mark.parametrize("path", ["lazy", "stream"])
-def test_c3_bert_base_fc2_full_size_twelve_layers(path, monkeypatch):
-    if path == "stream":
-        monkeypatch.setenv("ZIPLM_NEURON_PATH", "stream")
+def test_c3_bert_base_fc2_full_size_twelve_layers(path, neuron_variant):
+    neuron_variant(path)
     shape = wl.CONFIGS["c3_bert_base_fc2"][0]
     checked = [0, 7]
     W, H_or, out = run_full(shape, checked)

@@ -127,6 +127,33 @@ def test_hessian_streamed_batch_by_batch(dtype):
         assert err < 2e-6, err
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_device_stays_usable():
+    """The Hessian kernel's producer is given a poll limit of one look for its wait on a free
+    pipeline stage: on a healthy input with more K blocks than stages it gives up, every role
+    leaves through the abort path (issued copies and MMAs complete inside the live CTA, tensor
+    memory is freed), H[l][0][0] comes back NaN and the next stage reports ZIPLM_ERR_NONFINITE.
+    Nothing faults and nothing hangs; the same call works again with the default limit."""
+    z = zb()
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=64, d_latent=16, n_tokens=2048, n_layers=2)
+    _, X = wl.make_layers(sh, "cpu")
+    Xd = X.cuda()
+    z.set_option(z.Option.SPIN_LIMIT, 1)
+    try:
+        H = z.hessian_accumulate(Xd)
+        torch.cuda.synchronize()
+    finally:
+        z.set_option(z.Option.SPIN_LIMIT, 0)
+    assert torch.isnan(H[:, 0, 0]).all()
+    _, status = z.damped_inverse(H, 0.01)
+    torch.cuda.synchronize()
+    assert status.tolist() == [int(z.Status.ERR_NONFINITE)] * 2
+    H = z.hessian_accumulate(Xd)
+    torch.cuda.synchronize()
+    Ho = zo.hessian(X[1])
+    scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
+    assert np.max(np.abs(H[1].cpu().double().numpy() - Ho) / scale) < 2e-6
+
+
 def test_hessian_tokens_bad_args():
     z = zb()
     H = torch.ones(1, 8, 8, device="cuda")
@@ -196,13 +223,13 @@ def test_not_positive_definite_layer_is_flagged_and_others_finish():
 
 # ------------------------------------------------------------------ neuron path (a4 - a10)
 @pytest.fixture(params=["lazy", "stream"])
-def neuron_path(request, monkeypatch):
+def neuron_path(request):
     """Run a test once per neuron-path variant: delayed rank-B updates (default where the shape
     allows it) and the per-step streaming update."""
-    monkeypatch.delenv("ZIPLM_NEURON_PATH", raising=False)
-    if request.param == "stream":
-        monkeypatch.setenv("ZIPLM_NEURON_PATH", "stream")
-    return request.param
+    z = zb()
+    z.set_option(z.Option.NEURON_PATH, 1 if request.param == "stream" else 0)
+    yield request.param
+    z.set_option(z.Option.NEURON_PATH, 0)
 
 
 def test_c1_tiny_ffn_full_config(neuron_path):
@@ -232,6 +259,19 @@ def test_neuron_path_mid_size_full_depth_three_layers(neuron_path):
     print(reports)
 
 
+@pytest.mark.parametrize("d,check", [(1536, [0, 1]), (2048, [1])])
+def test_clustered_steps_kernel_full_depth_every_step(d, check):
+    """Full greedy order d -> 0 of the default path in lock-step with the oracle at widths where
+    the steps kernel runs on clusters of 2 (769..1536 live positions) and 4 (1537..2048) CTAs, and
+    on one CTA from 768 down: every single pick is compared, and every level's snapshot and loss."""
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=d, d_row=256, d_latent=d // 4,
+                   n_tokens=2 * d, n_layers=2, levels=tuple(range(d - d // 8, -1, -d // 8)))
+    out, reports = run_case(sh, check_layers=check)
+    for rep in reports:
+        assert rep["steps"] == d
+    print(reports)
+
+
 def test_neuron_path_is_deterministic(neuron_path):
     z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=256, d_row=64, d_latent=64,
@@ -246,7 +286,7 @@ def test_neuron_path_is_deterministic(neuron_path):
 
 
 @pytest.mark.parametrize("groups", ["1", "3", "8"])
-def test_layer_groups_do_not_change_the_result(groups, monkeypatch):
+def test_layer_groups_do_not_change_the_result(groups):
     """Layers are independent problems: how many groups of them run on internal streams must not
     change a single bit of any output."""
     z = zb()
@@ -254,12 +294,15 @@ def test_layer_groups_do_not_change_the_result(groups, monkeypatch):
                    n_tokens=1280, n_layers=9, levels=(256, 100, 0))
     W, X = wl.make_layers(sh, "cpu")
     H = torch.stack([oracle_h32(X[l]) for l in range(9)]).cuda()
-    monkeypatch.delenv("ZIPLM_LAYER_GROUPS", raising=False)
+    z.set_option(z.Option.LAYER_GROUPS, 0)
     ref = z.prune_layers(W.cuda(), H, 1, 0.01, [256, 100, 0])
     torch.cuda.synchronize()
-    monkeypatch.setenv("ZIPLM_LAYER_GROUPS", groups)
-    got = z.prune_layers(W.cuda(), H, 1, 0.01, [256, 100, 0])
-    torch.cuda.synchronize()
+    z.set_option(z.Option.LAYER_GROUPS, int(groups))
+    try:
+        got = z.prune_layers(W.cuda(), H, 1, 0.01, [256, 100, 0])
+        torch.cuda.synchronize()
+    finally:
+        z.set_option(z.Option.LAYER_GROUPS, 0)
     assert torch.count_nonzero(got["layer_status"]) == 0
     for k in ("order", "W_snap", "loss", "base_loss", "saliency"):
         assert torch.equal(ref[k], got[k]), k
@@ -298,17 +341,19 @@ def test_c2_bert_base_attention_shape_three_layers():
     run_case(sh, layers=[0, 5, 11])
 
 
-def test_block_path_with_group_size_one_agrees_with_neuron_path(monkeypatch, neuron_path):
+def test_block_path_with_group_size_one_agrees_with_neuron_path(neuron_path):
     z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=128, d_row=40, d_latent=32,
                    n_tokens=600, n_layers=2, levels=(128, 64, 0))
     W, X = wl.make_layers(sh, "cpu")
     H = torch.stack([oracle_h32(X[l]) for l in range(2)])
     a = z.prune_layers(W.cuda(), H.cuda(), 1, 0.01, [128, 64, 0])
-    monkeypatch.setenv("ZIPLM_FORCE_BLOCK_PATH", "1")
-    b = z.prune_layers(W.cuda(), H.cuda(), 1, 0.01, [128, 64, 0])
-    torch.cuda.synchronize()
-    monkeypatch.delenv("ZIPLM_FORCE_BLOCK_PATH")
+    z.set_option(z.Option.FORCE_BLOCK_PATH, 1)
+    try:
+        b = z.prune_layers(W.cuda(), H.cuda(), 1, 0.01, [128, 64, 0])
+        torch.cuda.synchronize()
+    finally:
+        z.set_option(z.Option.FORCE_BLOCK_PATH, 0)
     assert torch.equal(a["order"], b["order"])
     assert torch.allclose(a["W_snap"], b["W_snap"], rtol=1e-4, atol=1e-7)
     assert torch.allclose(a["loss"], b["loss"], rtol=1e-4)

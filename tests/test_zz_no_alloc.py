@@ -12,6 +12,7 @@ import pytest
 import torch
 
 import workloads as wl
+from oracle import ziplm_oracle as zo
 
 pytestmark = pytest.mark.gpu
 
@@ -41,6 +42,11 @@ def test_noalloc_inverse_matches_the_workspace_version_twice_in_a_row():
         Hl = Hl + float(np.float32(0.01)) * np.mean(np.diag(Hl)) * np.eye(d)
         tol = 50 * np.linalg.cond(Hl) * 2.2e-16
         assert np.max(np.abs(g - r)) / np.max(np.abs(r)) < tol
+        # and directly against the float64 oracle, layer by layer
+        for l in range(L):
+            Hd = zo.damped(H[l].cpu().numpy(), float(np.float32(0.01)))[0]
+            ref64 = zo.inverse_spd(Hd)
+            assert np.max(np.abs(g[l] - ref64)) / np.max(np.abs(ref64)) < 50 * np.linalg.cond(Hd) * 2.2e-16
 
 
 def test_noalloc_inverse_rejects_requests_beyond_its_scratch():
