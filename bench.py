@@ -169,20 +169,17 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in prune_lazy.cu)
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu captures
-# summarised under profiles/ (taken on 4 of the 12 layers and scaled by 3: traffic grows in
-# proportion to the layers).  Only valid for the bench workload; the kernels have not changed
-# since the captures.
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch: constants from earlier
+# ncu captures of these kernels (taken on 4 of the 12 layers and scaled by 3: traffic grows in
+# proportion to the layers), not measurements of this run.  Only valid for the bench workload.
 NCU_TRAFFIC = {
-    # k_lazy_update_aq, first block at full size (12 layers, n_new = 3040):
-    # profiles/k_lazy_update_aq_c3_12layers_every_launch.md
+    # k_lazy_update_aq, first block at full size (12 layers, n_new = 3040)
     "k_lazy_update_aq": dict(bytes=523.1e6 + 826.2e6, launch="n_new = 3040, m = 32, 12 layers",
                              algorithmic=12 * 24.0 * 3040 * 3039 / 2),
-    # k_dgemm_tiles, top-level product F21 = A21 M11^T: profiles/inverse_kernels_c3.md
+    # k_dgemm_tiles, top-level product F21 = A21 M11^T
     "k_dgemm_tiles": dict(bytes=3 * (116.6e6 + 49.0e6), launch="F21 = A21 M11^T, 12 x 24 macro tiles",
                           algorithmic=None),
-    # k_neuron_update, first step at full size (12 layers, n = 3071):
-    # profiles/k_neuron_update_c3_12layers_every_step.md
+    # k_neuron_update, first step at full size (12 layers, n = 3071)
     "k_neuron_update": dict(bytes=343.1e6 + 281.9e6, launch="n = 3071, 12 layers",
                             algorithmic=12 * (8.0 * 768 * 3071 + 4.0 * 3071 * 3071)),
 }
@@ -518,6 +515,64 @@ def run_ours(args, shape):
                            "float64 add + compare against a shared-memory value row")
         del mask, vals
 
+    # ---- the other workload families, one timed pass each (Hessian and pruning separately): the
+    # head path on BERT-base / BERT-large / GPT-2 attention shapes, BERT-large fc2, and the GPT-2
+    # shapes from 131072 bf16 tokens
+    others = None
+    if not args.skip_extras and rank == 0:
+        others = {}
+        del X, H, h_ws, p_ws
+        torch.cuda.empty_cache()
+        for fam, idx in (("c2_bert_base_attn", 0), ("c4_bert_large", 0), ("c4_bert_large", 1),
+                         ("c5_gpt2", 0), ("c5_gpt2", 1)):
+            sh = wl.CONFIGS[fam][idx]
+            Wo = torch.stack([wl.make_weight(sh, l) for l in range(sh.n_layers)]).to(dev)
+            Xo = torch.stack([wl.make_activations(sh, l, dev) for l in range(sh.n_layers)])
+            torch.cuda.synchronize()
+            lv = list(sh.levels)
+            Ho = torch.empty(sh.n_layers, sh.d_col, sh.d_col, dtype=torch.float32, device=dev)
+
+            def hess():
+                z.hessian_accumulate(Xo, Ho, alpha=2.0, beta=0.0)
+
+            res = [None]
+
+            def prune():
+                res[0] = z.prune_layers(Wo, Ho, sh.group_size, sh.damp_frac, lv, out=res[0])
+
+            t = {}
+            for nm, fn in (("hessian_ms", hess), ("prune_ms", prune)):
+                fn()
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(2):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                t[nm] = e0.elapsed_time(e1) / 2
+            assert int(torch.count_nonzero(res[0]["layer_status"])) == 0
+            z.set_option(z.Option.LAYER_GROUPS, 1)
+            z.profile_begin()
+            prune()
+            torch.cuda.synchronize()
+            ph = z.profile_end()
+            z.set_option(z.Option.LAYER_GROUPS, 0)
+            removed = sh.n_layers * (sh.n_groups - min(lv))
+            tot = t["hessian_ms"] + t["prune_ms"]
+            esz = 2 if sh.x_dtype != "f32" else 4
+            tri_flop = float(sh.n_layers) * sh.d_col * sh.d_col * sh.n_tokens      # lower triangle
+            others[sh.name] = dict(
+                layers=sh.n_layers, d_row=sh.d_row, d_col=sh.d_col, n_tokens=sh.n_tokens,
+                group_size=sh.group_size, x_dtype=sh.x_dtype, levels=len(lv),
+                hessian_ms=t["hessian_ms"], prune_ms=t["prune_ms"],
+                structures_per_sec=removed / (tot * 1e-3), layers_per_sec=sh.n_layers / (tot * 1e-3),
+                prune_structures_per_sec=removed / (t["prune_ms"] * 1e-3),
+                hessian_useful_tflops=tri_flop / (t["hessian_ms"] * 1e-3) / 1e12,
+                hessian_x_gb_per_s=sh.n_layers * sh.d_col * sh.n_tokens * esz / (t["hessian_ms"] * 1e-3) / 1e9,
+                phases_ms={k: round(v[0], 3) for k, v in ph.items() if v[1] > 0})
+            del Wo, Xo, Ho, res
+            torch.cuda.empty_cache()
+
     from paper_2302_04089_b200.parallel import max_over_ranks
     ms, ms_e2e = max_over_ranks(ms), max_over_ranks(ms_e2e)
     n_removed = G - min(levels)
@@ -541,6 +596,9 @@ def run_ours(args, shape):
         aq_bytes, aq_fma, _ = lazy_update_work(L, G, levels)
         aq_gbs = aq_bytes / (aq_ms * 1e-3) / 1e9 if aq_ms > 0 else 0.0
         fma_peak = 35.7                                # fp32 TFMA/s measured with a register-only FMA loop
+        hs_ms, _ = phases.get("hessian", (0.0, 0))
+        hs_useful = float(L) * d * d * N                      # lower triangle: d^2 N flop per layer
+        tf32_peak = 1115.0    # TFLOP/s: tcgen05.mma kind::tf32, M = 128, N >= 128, operands in shared memory
         line = dict(
             metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
             warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
@@ -589,6 +647,19 @@ def run_ours(args, shape):
                                    note="3 fp32 FMA per entry and pending step; peak = measured "
                                         "71.4 TFLOP/s fp32 (nominal 148 SMs x 128 lanes x 1.965 GHz "
                                         "= 74.4)")),
+            roofline_hessian=dict(
+                kernel="k_split_tf32 + k_syrk_tc<tf32>", bound="tensor",
+                achieved=3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0, peak=tf32_peak,
+                unit="TFLOP/s", frac=(3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 / tf32_peak) if hs_ms > 0 else 0.0,
+                useful_tflops=hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0,
+                traffic=None, ms=hs_ms,
+                peak_source="measured on this part: one thread per SM issuing tcgen05.mma kind::tf32 "
+                            "128 x 128 x 8 back to back from shared-memory operands, 1114 TFLOP/s at "
+                            "N = 128 and 1116 at N = 256 (735 at N = 64; kind::f16 bf16 the same way: "
+                            "2225); nominal 1.1 PFLOP/s",
+                note="fp32 activations: every product is three TF32 MMAs (hi*hi, hi*lo, lo*hi), so "
+                     "the tensor-pipe work is 3 x the useful d^2 N flop per layer; the time is that "
+                     "of the whole call, the split pre-pass included"),
             roofline_streaming_update=dict(
                 kernel="k_neuron_update", bound="hbm", achieved=achieved, peak=peak, unit="GB/s",
                 frac=achieved / peak,
@@ -608,6 +679,12 @@ def run_ours(args, shape):
             line["reshape_database"] = reshape
         if select is not None:
             line["level_selection"] = select
+        if others is not None:
+            line["other_workloads"] = others
+            line["other_workloads_note"] = (
+                "one call each, inputs resident, mean of 2 after 1 warm-up; hessian_useful_tflops "
+                "counts d^2 N flop per layer (the lower triangle); phases_ms from one more pruning "
+                "call with the layer groups run back to back")
         if world == 1 and not args.no_cpu_baseline:
             s = oracle_sample(shape, n_loop_steps=args.oracle_steps)
             line["cpu_baseline"] = dict(
