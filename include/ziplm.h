@@ -188,7 +188,7 @@ ziplm_status ziplm_damped_inverse_noalloc(const float* H, int L, int d, float da
  *   W            dev, [L, d_row, d_col] fp32; not modified
  *   H            dev, [L, d_col, d_col] fp32, the UNDAMPED 2 X X^T, symmetric; not modified;
  *                16-byte aligned (ZIPLM_ERR_INVALID_ARG otherwise)
- *   group_size   columns per structure; d_col % group_size == 0; 1 <= group_size <= 64
+ *   group_size   columns per structure; d_col % group_size == 0; 1 <= group_size <= 128
  *   damp_frac    lambda = damp_frac * mean(diag H[l]); >= 0
  *   levels       HOST, [n_levels] numbers of REMAINING structures, strictly decreasing, each in
  *                [0, G]; level 0 removes the whole module, level G is the unpruned layer
@@ -206,7 +206,7 @@ ziplm_status ziplm_damped_inverse_noalloc(const float* H, int L, int d, float da
  * of the damped least-squares objective; it needs no extra pass over H.
  *
  * Errors: ZIPLM_ERR_INVALID_ARG (shapes, NULL pointers, levels not strictly decreasing or out
- * of range, damp_frac < 0 or not finite), ZIPLM_ERR_UNSUPPORTED (group_size > 64),
+ * of range, damp_frac < 0 or not finite), ZIPLM_ERR_UNSUPPORTED (group_size > 128),
  * ZIPLM_ERR_WORKSPACE, ZIPLM_ERR_CUDA.
  */
 size_t ziplm_prune_workspace_bytes(int L, int d_row, int d_col, int group_size, int n_levels);

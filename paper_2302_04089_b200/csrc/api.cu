@@ -106,7 +106,7 @@ ziplm_status ziplm_damped_inverse(const float* H, int L, int d, float damp_frac,
 
 size_t ziplm_prune_workspace_bytes(int L, int d_row, int d_col, int group_size, int n_levels) {
     if (L < 1 || d_row < 1 || d_col < 1 || group_size < 1 || n_levels < 0) return 0;
-    if (d_col % group_size != 0 || group_size > 64) return 0;
+    if (d_col % group_size != 0 || group_size > 128) return 0;
     if (group_size == 1 && !force_block_path())
         return neuron_workspace_bytes(L, d_row, d_col, n_levels);
     return block_workspace_bytes(L, d_row, d_col, group_size, n_levels);
@@ -128,7 +128,7 @@ ziplm_status ziplm_prune_layers(const float* W, const float* H, int L, int d_row
         if (levels[i] < 0 || levels[i] > G) return ZIPLM_ERR_INVALID_ARG;
         if (i > 0 && levels[i] >= levels[i - 1]) return ZIPLM_ERR_INVALID_ARG;
     }
-    if (group_size > 64) return ZIPLM_ERR_UNSUPPORTED;
+    if (group_size > 128) return ZIPLM_ERR_UNSUPPORTED;
     const size_t need = ziplm_prune_workspace_bytes(L, d_row, d_col, group_size, n_levels);
     if (!workspace || !aligned(workspace, kAlign) || workspace_bytes < need) return ZIPLM_ERR_WORKSPACE;
     if (!have_device()) return ZIPLM_ERR_CUDA;

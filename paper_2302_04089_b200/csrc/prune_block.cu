@@ -19,7 +19,7 @@
 namespace ziplm {
 namespace {
 
-constexpr int GMAX = 64;
+constexpr int GMAX = 128;     // widest structure; kernels are instantiated for 64 and 128
 
 struct BlockState {
     int chosen;      // structure selected in the current step
@@ -28,9 +28,10 @@ struct BlockState {
     double dw2;      // scratch: ||W - W_snap||_F^2 of the snapshot being written
 };
 
-// In-place lower Cholesky of the g x g matrix in s (row pitch GMAX + 1), all threads of the block.
+// In-place lower Cholesky of the g x g matrix in s (row pitch GM + 1), all threads of the block.
 // Returns through *flag a ziplm_status if a pivot is not positive / not finite.
-__device__ void chol_smem(double (*s)[GMAX + 1], int g, int* flag) {
+template <int GM>
+__device__ void chol_smem(double (*s)[GM + 1], int g, int* flag) {
     const int tid = threadIdx.x, nt = blockDim.x;
     for (int c = 0; c < g; ++c) {
         if (tid == 0) {
@@ -66,13 +67,16 @@ __global__ void k_block_init_state(int L, int G, BlockState* __restrict__ state,
     if (i < L * G) alive[i] = 1;
 }
 
-// rho_S for every live structure: one block per (structure, layer).
+// rho_S for every live structure: one block per (structure, layer).  The g x g block lives in
+// dynamic shared memory ((GM + 1) * g doubles), GM = 64 or 128 bounding g.
+template <int GM>
 __global__ void __launch_bounds__(256) k_block_score(int r, int d, int g, int G,
                                                      const double* __restrict__ A,
                                                      const double* __restrict__ W64,
                                                      const int* __restrict__ alive,
                                                      double* __restrict__ rho, int* layer_status) {
-    __shared__ double sB[GMAX][GMAX + 1];
+    extern __shared__ double dyn_block[];
+    double (*sB)[GM + 1] = reinterpret_cast<double (*)[GM + 1]>(dyn_block);
     __shared__ double red[8];
     __shared__ int flag;
     const int l = blockIdx.y, s = blockIdx.x;
@@ -84,10 +88,10 @@ __global__ void __launch_bounds__(256) k_block_score(int r, int d, int g, int G,
     if (tid == 0) flag = 0;
     for (int e = tid; e < g * g; e += 256) sB[e / g][e % g] = Al[(size_t)(c0 + e / g) * d + c0 + e % g];
     __syncthreads();
-    chol_smem(sB, g, &flag);
+    chol_smem<GM>(sB, g, &flag);
     double acc = 0.0;
     for (int i = tid; i < r; i += 256) {
-        double y[GMAX];
+        double y[GM];
         const double* w = Wl + (size_t)i * d + c0;
         for (int k = 0; k < g; ++k) {
             double v = w[k];
@@ -149,12 +153,14 @@ __global__ void __launch_bounds__(256) k_block_select(int G, int t, const double
 }
 
 // Q = C_B^-1 [ (H^-1)[S,:] | W[:,S]^T ]  (gp x (d + r), rows >= g zero) for the selected structure.
+template <int GM>
 __global__ void __launch_bounds__(256) k_block_solve(int r, int d, int g, int gp,
                                                      const double* __restrict__ A,
                                                      const double* __restrict__ W64,
                                                      const BlockState* __restrict__ state,
                                                      double* __restrict__ Q) {
-    __shared__ double sB[GMAX][GMAX + 1];
+    extern __shared__ double dyn_block[];
+    double (*sB)[GM + 1] = reinterpret_cast<double (*)[GM + 1]>(dyn_block);
     __shared__ int flag;
     const int l = blockIdx.y, tid = threadIdx.x;
     const double* Al = A + (size_t)l * d * d;
@@ -164,10 +170,10 @@ __global__ void __launch_bounds__(256) k_block_solve(int r, int d, int g, int gp
     if (tid == 0) flag = 0;
     for (int e = tid; e < g * g; e += 256) sB[e / g][e % g] = Al[(size_t)(c0 + e / g) * d + c0 + e % g];
     __syncthreads();
-    chol_smem(sB, g, &flag);
+    chol_smem<GM>(sB, g, &flag);
     const int j = blockIdx.x * 256 + tid;
     if (j >= d + r) return;
-    double y[GMAX];
+    double y[GM];
     for (int k = 0; k < g; ++k) {
         double v = (j < d) ? Al[(size_t)(c0 + k) * d + j] : Wl[(size_t)(j - d) * d + c0 + k];
         for (int m = 0; m < k; ++m) v -= sB[k][m] * y[m];
@@ -336,6 +342,14 @@ ziplm_status run_prune_blocks(const float* W, const float* H, int L, int r, int 
         return ZIPLM_OK;
     };
 
+    // the g x g block of the score and solve kernels: g rows of GM + 1 doubles
+    const size_t blk_smem = sizeof(double) * (size_t)g * ((g <= 64 ? 64 : 128) + 1);
+    if (g > 64) {
+        ZIPLM_CHECK_CUDA(cudaFuncSetAttribute(k_block_score<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)blk_smem));
+        ZIPLM_CHECK_CUDA(cudaFuncSetAttribute(k_block_solve<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)blk_smem));
+    }
     int n = G, slot = 0;
     if (slot < n_levels && levels[slot] == n) {
         s = snapshot(slot++);
@@ -345,8 +359,12 @@ ziplm_status run_prune_blocks(const float* W, const float* H, int L, int r, int 
     for (int t = 0; n > n_min; ++t) {
         {
             PhaseScope ps(PH_BLOCK_SCORE, st);
-            k_block_score<<<dim3(G, L), 256, 0, st>>>(r, d, g, G, w.A, w.W64, w.alive, w.rho,
-                                                     layer_status);
+            if (g <= 64)
+                k_block_score<64><<<dim3(G, L), 256, blk_smem, st>>>(r, d, g, G, w.A, w.W64, w.alive, w.rho,
+                                                                     layer_status);
+            else
+                k_block_score<128><<<dim3(G, L), 256, blk_smem, st>>>(r, d, g, G, w.A, w.W64, w.alive, w.rho,
+                                                                      layer_status);
             ZIPLM_CHECK_LAUNCH();
             k_block_select<<<L, 256, 0, st>>>(G, t, w.rho, w.alive, w.state, order, saliency,
                                               layer_status);
@@ -354,8 +372,12 @@ ziplm_status run_prune_blocks(const float* W, const float* H, int L, int r, int 
         }
         if (n > 1) {
             PhaseScope ps(PH_BLOCK_UPDATE, st);
-            k_block_solve<<<dim3((d + r + 255) / 256, L), 256, 0, st>>>(r, d, g, w.gp, w.A, w.W64,
-                                                                       w.state, w.Q);
+            if (g <= 64)
+                k_block_solve<64><<<dim3((d + r + 255) / 256, L), 256, blk_smem, st>>>(r, d, g, w.gp, w.A, w.W64,
+                                                                                      w.state, w.Q);
+            else
+                k_block_solve<128><<<dim3((d + r + 255) / 256, L), 256, blk_smem, st>>>(r, d, g, w.gp, w.A, w.W64,
+                                                                                       w.state, w.Q);
             ZIPLM_CHECK_LAUNCH();
             k_block_update<<<dim3((d + 63) / 64, (d + r + 63) / 64, L), 256, 0, st>>>(r, d, w.gp, w.A,
                                                                                      w.W64, w.Q);

@@ -328,6 +328,11 @@ def test_workspace_is_not_assumed_clean(neuron_path):
     (96, 2, 20, 2, [48, 40, 17, 0]),            # tiny groups, many steps
     (120, 24, 33, 1, [4, 1]),                   # group size that is no power of two, ragged rows
     (192, 64, 200, 3, [2]),
+    (512, 128, 96, 2, [4, 3, 2, 1, 0]),         # 128-wide heads: four structures, every head count
+    (1024, 128, 160, 2, [8, 6, 3, 0]),          # eight 128-wide heads
+    (768, 96, 64, 1, [8, 5, 0]),                # width between 64 and 128
+    (1024, 128, 256, 2, [8, 7, 4, 1]),          # grouped-query shape: out-projection input of 8
+                                                # heads of width 128 feeding a narrow output
 ])
 def test_block_path_small_shapes(d, g, r, L, levels):
     sh = wl.scaled(wl.CONFIGS["c2_bert_base_attn"][0], d_col=d, d_row=r, group_size=g,

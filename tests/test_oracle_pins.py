@@ -97,7 +97,7 @@ def test_hand_worked_group_fixture():
 
 # ------------------------------------------------------------------ brute force (Eq. 2, Eq. 3)
 @pytest.mark.parametrize("d,g,r,seed", [(6, 1, 3, 0), (8, 2, 4, 1), (12, 3, 5, 2), (9, 1, 2, 3),
-                                        (10, 2, 1, 4)])
+                                        (10, 2, 1, 4), (16, 4, 3, 5)])
 def test_every_greedy_step_against_brute_force_refit(d, g, r, seed):
     """Eq. 2 is the increase of the (damped) least-squares error when S is removed and the
     survivors are refitted; Eq. 3 is that refit.  Checked for EVERY candidate at EVERY step."""
