@@ -222,6 +222,8 @@ def run_ours(args, shape):
     from paper_2302_04089_b200 import build as zbuild
     zbuild.build()
 
+    if args.layer_groups:
+        z.set_option(z.Option.LAYER_GROUPS, args.layer_groups)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -384,7 +386,7 @@ def run_ours(args, shape):
         torch.cuda.synchronize()
         phases_stream = z.profile_end()
         z.set_option(z.Option.NEURON_PATH, 0)
-    z.set_option(z.Option.LAYER_GROUPS, 0)
+    z.set_option(z.Option.LAYER_GROUPS, args.layer_groups)
 
     # ---- the Hessian from token-major activations (one token per row, the layout a forward pass
     # emits): one call on the whole calibration set, and eight calibration batches with beta = 1
@@ -556,7 +558,7 @@ def run_ours(args, shape):
             prune()
             torch.cuda.synchronize()
             ph = z.profile_end()
-            z.set_option(z.Option.LAYER_GROUPS, 0)
+            z.set_option(z.Option.LAYER_GROUPS, args.layer_groups)
             removed = sh.n_layers * (sh.n_groups - min(lv))
             tot = t["hessian_ms"] + t["prune_ms"]
             esz = 2 if sh.x_dtype != "f32" else 4
@@ -709,6 +711,9 @@ def main():
                     help="profiling aid: use only this many of the workload's layers")
     ap.add_argument("--max-removed", type=int, default=0,
                     help="profiling aid: stop the greedy loop after this many removals")
+    ap.add_argument("--layer-groups", type=int, default=0,
+                    help="profiling aid: number of layer groups on internal streams (0 = library default; "
+                         "1 runs them back to back, so that a profiler's per-kernel times add up)")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling aid: no host-buffer leg")
     ap.add_argument("--skip-extras", action="store_true",
                     help="profiling aid: no token-major Hessian / reshaping / level-selection legs")
