@@ -113,6 +113,141 @@ __global__ void __launch_bounds__(256) k_block_score(int r, int d, int g, int G,
     }
 }
 
+// rho_S for structures of up to 64 columns without a dependent chain per weight row:
+//     rho_S = tr(W[:,S] B^-1 W[:,S]^T) = < C_B^-1 G_S , C_B^-1 >_F ,   G_S = W[:,S]^T W[:,S]
+// One block per (structure, layer): Cholesky of B, the g x g Gram block of the structure's weight
+// columns as a register-tiled product over the d_row rows, the inverse of the factor (one thread
+// per column), the g x g product and the reduction -- all in float64.  The inverse of the factor
+// is also written to Cinv[l][s] for the solve kernel of the structure that gets selected.
+// Dynamic shared memory: three g x 65 matrices and a 32 x 65 staging tile.
+constexpr int GS = 64;                         // widest structure of this kernel
+constexpr size_t kScoreGramSmem = sizeof(double) * (3 * GS + 32) * (GS + 1);
+__global__ void __launch_bounds__(256) k_block_score_gram(int r, int d, int g, int G,
+                                                          const double* __restrict__ A,
+                                                          const double* __restrict__ W64,
+                                                          const int* __restrict__ alive,
+                                                          double* __restrict__ rho,
+                                                          double* __restrict__ Cinv, int* layer_status) {
+    extern __shared__ double dyn_block[];
+    double (*sB)[GS + 1] = reinterpret_cast<double (*)[GS + 1]>(dyn_block);                  // B, then C
+    double (*sG)[GS + 1] = reinterpret_cast<double (*)[GS + 1]>(dyn_block + GS * (GS + 1));  // Gram block
+    double (*sI)[GS + 1] = reinterpret_cast<double (*)[GS + 1]>(dyn_block + 2 * GS * (GS + 1));  // C^-1
+    double (*sW)[GS + 1] = reinterpret_cast<double (*)[GS + 1]>(dyn_block + 3 * GS * (GS + 1));  // 32 rows of W
+    __shared__ double red[8];
+    __shared__ int flag;
+    const int l = blockIdx.y, s = blockIdx.x;
+    if (!alive[(size_t)l * G + s]) return;
+    const int tid = threadIdx.x;
+    const double* Al = A + (size_t)l * d * d;
+    const double* Wl = W64 + (size_t)l * r * d;
+    const int c0 = s * g;
+    if (tid == 0) flag = 0;
+    for (int e = tid; e < g * g; e += 256) sB[e / g][e % g] = Al[(size_t)(c0 + e / g) * d + c0 + e % g];
+    // Gram block: thread (ty, tx) owns entries (4 ty + a, 4 tx + b); rows of W staged 32 at a time
+    const int ty = tid >> 4, tx = tid & 15;
+    double acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+    for (int i0 = 0; i0 < r; i0 += 32) {
+        __syncthreads();
+        for (int e = tid; e < 32 * g; e += 256) {
+            const int ii = e / g, k = e % g;
+            sW[ii][k] = (i0 + ii < r) ? Wl[(size_t)(i0 + ii) * d + c0 + k] : 0.0;
+        }
+        __syncthreads();
+        if (4 * ty < g && 4 * tx < g) {
+#pragma unroll 4
+            for (int ii = 0; ii < 32; ++ii) {
+                double wa[4], wb[4];
+#pragma unroll
+                for (int a = 0; a < 4; ++a) { wa[a] = sW[ii][4 * ty + a]; wb[a] = sW[ii][4 * tx + a]; }
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) acc[a][b] = fma(wa[a], wb[b], acc[a][b]);
+            }
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+            if (4 * ty + a < g && 4 * tx + b < g) sG[4 * ty + a][4 * tx + b] = acc[a][b];
+    __syncthreads();
+    chol_smem<GS>(sB, g, &flag);
+    // C^-1, one thread per column j: column j of the inverse of a lower triangular matrix
+    if (tid < g) {
+        const int j = tid;
+        for (int k = 0; k < j; ++k) sI[k][j] = 0.0;
+        for (int k = j; k < g; ++k) {
+            double v = (k == j) ? 1.0 : 0.0;
+            for (int m = j; m < k; ++m) v -= sB[k][m] * sI[m][j];
+            sI[k][j] = v / sB[k][k];
+        }
+    }
+    __syncthreads();
+    // rho = sum_{k,j} (C^-1 G)[k][j] * C^-1[k][j]; C^-1 is lower triangular
+    double part = 0.0;
+    for (int e = tid; e < g * g; e += 256) {
+        const int k = e / g, j = e % g;
+        if (j > k) continue;
+        double t = 0.0;
+        for (int m = 0; m <= k; ++m) t = fma(sI[k][m], sG[m][j], t);
+        part = fma(t, sI[k][j], part);
+    }
+    double* Ci = Cinv + ((size_t)l * G + s) * g * g;
+    for (int e = tid; e < g * g; e += 256) Ci[e] = sI[e / g][e % g];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if ((tid & 31) == 0) red[tid >> 5] = part;
+    __syncthreads();
+    if (tid == 0) {
+        double t = 0.0;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        rho[(size_t)l * G + s] = t;
+        if (flag) set_layer_status(layer_status, l, flag);
+    }
+}
+
+// Q = C_B^-1 [ (H^-1)[S,:] | W[:,S]^T ] for the selected structure from the stored inverse factor:
+// a plain product, one column per thread (g <= 64).
+__global__ void __launch_bounds__(256) k_block_solve_inv(int r, int d, int g, int gp, int G,
+                                                         const double* __restrict__ A,
+                                                         const double* __restrict__ W64,
+                                                         const double* __restrict__ Cinv,
+                                                         const BlockState* __restrict__ state,
+                                                         double* __restrict__ Q) {
+    __shared__ double sI[GS * (GS + 1) / 2];       // rows of the lower triangle, packed
+    const int l = blockIdx.y, tid = threadIdx.x;
+    const double* Al = A + (size_t)l * d * d;
+    const double* Wl = W64 + (size_t)l * r * d;
+    double* Ql = Q + (size_t)l * gp * (d + r);
+    const int chosen = state[l].chosen, c0 = chosen * g;
+    const double* Ci = Cinv + ((size_t)l * G + chosen) * g * g;
+    for (int e = tid; e < g * g; e += 256) {
+        const int k = e / g, m = e % g;
+        if (m <= k) sI[k * (k + 1) / 2 + m] = Ci[e];
+    }
+    __syncthreads();
+    const int j = blockIdx.x * 256 + tid;
+    if (j >= d + r) return;
+    double x[GS];
+#pragma unroll
+    for (int k = 0; k < GS; ++k)
+        x[k] = (k < g) ? ((j < d) ? Al[(size_t)(c0 + k) * d + j] : Wl[(size_t)(j - d) * d + c0 + k]) : 0.0;
+    for (int k = 0; k < g; ++k) {
+        const double* row = sI + k * (k + 1) / 2;
+        double v0 = 0.0, v1 = 0.0;
+        int m = 0;
+        for (; m + 1 <= k; m += 2) { v0 = fma(row[m], x[m], v0); v1 = fma(row[m + 1], x[m + 1], v1); }
+        if (m <= k) v0 = fma(row[m], x[m], v0);
+        Ql[(size_t)k * (d + r) + j] = v0 + v1;
+    }
+    for (int k = g; k < gp; ++k) Ql[(size_t)k * (d + r) + j] = 0.0;
+}
+
 // argmin over live structures (ties -> lowest index), bookkeeping.  One block per layer.
 __global__ void __launch_bounds__(256) k_block_select(int G, int t, const double* __restrict__ rho,
                                                       int* __restrict__ alive,
@@ -271,7 +406,7 @@ __global__ void k_block_loss(int L, int n_levels, int slot, const double* __rest
 }
 
 struct BlockWs {
-    double* A; double* W64; double* Q; double* rho; int* alive; BlockState* state; double* lam;
+    double* A; double* W64; double* Q; double* rho; double* Cinv; int* alive; BlockState* state; double* lam;
     double* base_acc; void* inv_ws; size_t inv_bytes; int gp; size_t total;
 };
 
@@ -284,6 +419,7 @@ BlockWs carve_block(void* ws, int L, int r, int d, int g) {
     w.W64 = c.take<double>((size_t)L * r * d);
     w.Q = c.take<double>((size_t)L * w.gp * (d + r));
     w.rho = c.take<double>((size_t)L * G);
+    w.Cinv = c.take<double>(g <= GS ? (size_t)L * G * g * g : 0);      // inverse factors (g <= 64)
     w.alive = c.take<int>((size_t)L * G);
     w.state = c.take<BlockState>((size_t)L);
     w.lam = c.take<double>((size_t)L);
@@ -344,6 +480,9 @@ ziplm_status run_prune_blocks(const float* W, const float* H, int L, int r, int 
 
     // the g x g block of the score and solve kernels: g rows of GM + 1 doubles
     const size_t blk_smem = sizeof(double) * (size_t)g * ((g <= 64 ? 64 : 128) + 1);
+    if (g <= GS)
+        ZIPLM_CHECK_CUDA(cudaFuncSetAttribute(k_block_score_gram, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kScoreGramSmem));
     if (g > 64) {
         ZIPLM_CHECK_CUDA(cudaFuncSetAttribute(k_block_score<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)blk_smem));
@@ -359,9 +498,9 @@ ziplm_status run_prune_blocks(const float* W, const float* H, int L, int r, int 
     for (int t = 0; n > n_min; ++t) {
         {
             PhaseScope ps(PH_BLOCK_SCORE, st);
-            if (g <= 64)
-                k_block_score<64><<<dim3(G, L), 256, blk_smem, st>>>(r, d, g, G, w.A, w.W64, w.alive, w.rho,
-                                                                     layer_status);
+            if (g <= GS)
+                k_block_score_gram<<<dim3(G, L), 256, kScoreGramSmem, st>>>(r, d, g, G, w.A, w.W64, w.alive,
+                                                                            w.rho, w.Cinv, layer_status);
             else
                 k_block_score<128><<<dim3(G, L), 256, blk_smem, st>>>(r, d, g, G, w.A, w.W64, w.alive, w.rho,
                                                                       layer_status);
@@ -372,9 +511,9 @@ ziplm_status run_prune_blocks(const float* W, const float* H, int L, int r, int 
         }
         if (n > 1) {
             PhaseScope ps(PH_BLOCK_UPDATE, st);
-            if (g <= 64)
-                k_block_solve<64><<<dim3((d + r + 255) / 256, L), 256, blk_smem, st>>>(r, d, g, w.gp, w.A, w.W64,
-                                                                                      w.state, w.Q);
+            if (g <= GS)
+                k_block_solve_inv<<<dim3((d + r + 255) / 256, L), 256, 0, st>>>(r, d, g, w.gp, G, w.A, w.W64,
+                                                                               w.Cinv, w.state, w.Q);
             else
                 k_block_solve<128><<<dim3((d + r + 255) / 256, L), 256, blk_smem, st>>>(r, d, g, w.gp, w.A, w.W64,
                                                                                        w.state, w.Q);
