@@ -641,9 +641,17 @@ def run_ours(args, shape):
                           traffic_note=NCU_TRAFFIC["k_lazy_update_aq"], peak_source=peak_src,
                           launches=aq_n, avg_launch_us=1e3 * aq_ms / max(aq_n, 1),
                           algorithmic_bytes_per_step=aq_bytes,
+                          symmetric=dict(bytes_per_step=aq_bytes * 16.0 / 24.0,
+                                         achieved=aq_gbs * 16.0 / 24.0, frac=aq_gbs * 16.0 / 24.0 / peak,
+                                         note="one read and one write per unique entry of the two "
+                                              "symmetric matrices (16 B per pair); the kernel's own "
+                                              "count (24 B) includes the second, mirrored store that "
+                                              "lets the steps kernel read a pivot column as a row"),
                           note="rank-32 update of H^-1 and Q, the kernel with the largest summed time "
-                               "in the timed path; it sits between the memory system and the fp32 "
-                               "issue rate (see alu)",
+                               "in the timed path; bound by its 4-byte gather through the compaction "
+                               "map (a stand-alone kernel with the same gather, mirror and direct "
+                               "stores and no arithmetic reaches 3.3-3.9 TB/s on this part, 4.7 with "
+                               "16-byte aligned reads), with the fp32 issue rate close behind (see alu)",
                           alu=dict(achieved_tfma=aq_fma / (aq_ms * 1e-3) / 1e12 if aq_ms > 0 else 0.0,
                                    peak_tfma=fma_peak,
                                    note="3 fp32 FMA per entry and pending step; peak = measured "
