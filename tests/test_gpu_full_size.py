@@ -235,7 +235,7 @@ def test_paper_database_grid_from_streamed_token_major_batches():
     Ho = zo.hessian(X[l])
     scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
     err = np.max(np.abs(H[l].cpu().double().numpy() - Ho) / scale)
-    assert err < hessian_tol("f32"), err
+    assert err < HESSIAN_TOL, err
     # eight batches and one pass differ only by the rounding of seven more fp32 additions
     H1 = z.hessian_accumulate(X[l:l + 1])
     assert torch.allclose(H[l], H1[0], rtol=0, atol=4e-6 * float(H1[0].diagonal().max()))
@@ -277,4 +277,4 @@ def test_paper_database_grid_from_streamed_token_major_batches():
         Ho = zo.hessian(X[l])
         scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
         err = np.max(np.abs(H[l].cpu().double().numpy() - Ho) / scale)
-        assert err < hessian_tol("bf16"), err
+        assert err < HESSIAN_TOL, err
