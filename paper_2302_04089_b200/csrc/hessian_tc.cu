@@ -8,9 +8,15 @@
 //
 //   bf16 / fp16 X : kind::f16 (both operands of the same 16-bit type, exact products, fp32
 //            accumulate), K block of 64 tokens.
-//   fp32 X : a pre-pass writes X_hi (fp32 with the 13 low mantissa bits cleared = a TF32 value)
-//            and X_lo = X - X_hi; the kernel accumulates hi*hi + hi*lo + lo*hi with kind::tf32,
-//            which keeps ~21 mantissa bits per product.  K block of 32 tokens.
+//   fp32 X : a pre-pass scales every feature row by a power of two s_i (so that its largest
+//            entry lies in [2^13, 2^14): the whole fp16 range is used whatever the row's
+//            magnitude) and writes two fp16 parts, X_1 = fp16(s x) and X_2 = fp16(s x - X_1);
+//            the kernel accumulates X_1 X_1^T + X_1 X_2^T + X_2 X_1^T with kind::f16 (exact
+//            products, fp32 accumulate), which keeps ~21 mantissa bits per product, and the
+//            epilogue multiplies entry (i, j) by 1 / (s_i s_j) (exact).  K block of 64 tokens:
+//            half the operand bytes and half the MMAs of a TF32 hi / lo split of the same
+//            accuracy, which matters because the kernel is bound by the L2 -> shared-memory
+//            operand traffic.
 //
 // One CTA per tile: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..9 =
 // epilogue (two per TMEM lane quarter; they drain the accumulator every few K blocks, see
@@ -21,6 +27,7 @@
 // a raised error word into NaN in H[l][0][0] of every layer.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 #include "tc_common.cuh"
@@ -33,8 +40,8 @@ constexpr int TM = 128;                 // tile rows / cols
 constexpr int ROW_BYTES = 128;          // one swizzle row
 constexpr int TILE_BYTES = TM * ROW_BYTES;   // 16 KiB per operand tile per K block
 
-template <bool TF32> struct Cfg;
-template <> struct Cfg<true>  { static constexpr int BK = 32, UK = 8,  STAGES = 3, TILES = 4; };
+template <bool SPLIT> struct Cfg;   // SPLIT: two fp16 parts per operand (fp32 inputs)
+template <> struct Cfg<true>  { static constexpr int BK = 64, UK = 16, STAGES = 3, TILES = 4; };
 template <> struct Cfg<false> { static constexpr int BK = 64, UK = 16, STAGES = 5, TILES = 2; };
 
 // Tensor-memory accumulators truncate when they add (measured: the error of a chain of S
@@ -42,19 +49,31 @@ template <> struct Cfg<false> { static constexpr int BK = 64, UK = 16, STAGES = 
 // accumulator is double-buffered, and after every CHUNK K blocks (8 MMAs) the epilogue warps
 // drain it into fp32 registers, where the partial sums are added with round-to-nearest in two
 // levels (a running sum that is folded into the total every FOLD drains, so that neither level
-// adds more than a few dozen terms).  The TF32 cross terms hi*lo + lo*hi are 2^-11 of the main
-// term; they get an accumulator of their own that is only read at the end, so their truncation
-// is negligible.
+// adds more than a few dozen terms).  The cross terms X_1 X_2^T + X_2 X_1^T of the split are
+// 2^-11 of the main term; they get an accumulator of their own that is only read at the end, so
+// their truncation is negligible.
 constexpr int CHUNK = 2;
 constexpr int FOLD = 32;
 constexpr int EPI_WARPS = 8;                  // two warps per TMEM lane quarter, 64 columns each
 constexpr int THREADS = 32 * (2 + EPI_WARPS);
 
+// Power-of-two scale of a feature row from the bit pattern of its largest magnitude m: the largest
+// scaled entry lies in [2^13, 2^14).  inverse = true gives 1 / scale.  Rows of zeros and
+// non-finite rows are left alone; the exponent is clamped so that the scale is a normal number.
+__device__ __forceinline__ float row_scale(unsigned amax_bits, bool inverse) {
+    const int e = (int)((amax_bits >> 23) & 255u);
+    if (amax_bits == 0u || e == 255) return 1.f;
+    int k = 140 - e;                       // m in [2^(e-127), 2^(e-126))  ->  m 2^k < 2^14
+    k = k > 100 ? 100 : (k < -100 ? -100 : k);
+    return __int_as_float((127 + (inverse ? -k : k)) << 23);
+}
+
 template <bool TF32>
 __global__ void __launch_bounds__(THREADS, 1)
 k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
           float* __restrict__ H, int d, int num_kb, float alpha, float beta, int layer0,
-          int* __restrict__ err_word, uint32_t fmt16, uint32_t empty_spin_limit) {
+          int* __restrict__ err_word, uint32_t fmt16, uint32_t empty_spin_limit,
+          const unsigned* __restrict__ amax) {
     using C = Cfg<TF32>;
     constexpr int STAGE_BYTES = C::TILES * TILE_BYTES;
     constexpr uint32_t TMEM_COLS = TF32 ? 512u : 256u;   // main x2 (+ cross terms), power of two
@@ -127,8 +146,8 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- MMA issuer
-            // operand format of the instruction: 2 = TF32; 16-bit inputs: 1 = BF16, 0 = F16 (A and B alike)
-            const uint32_t idesc = make_idesc(TF32 ? 2u : fmt16, TM, TM);
+            // operand format of the instruction: 1 = BF16, 0 = F16 (A and B alike; the split is fp16)
+            const uint32_t idesc = make_idesc(TF32 ? 0u : fmt16, TM, TM);
             const uint32_t tmem_cross = tmem_base + 256u;
             int kb = 0;
             for (int c = 0; c < num_chunks && !failed; ++c) {
@@ -157,9 +176,9 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
                         const uint64_t adv = (uint64_t)(k * 32 / 16);   // 32 bytes per MMA along K
                         const uint32_t acc_main = ((kb - kb_first) | k) ? 1u : 0u;
                         if (TF32) {
-                            umma_tf32(tmem_main, a_hi + adv, b_hi + adv, idesc, acc_main);
-                            umma_tf32(tmem_cross, a_hi + adv, b_lo + adv, idesc, (kb | k) ? 1u : 0u);
-                            umma_tf32(tmem_cross, a_lo + adv, b_hi + adv, idesc, 1u);
+                            umma_bf16(tmem_main, a_hi + adv, b_hi + adv, idesc, acc_main);
+                            umma_bf16(tmem_cross, a_hi + adv, b_lo + adv, idesc, (kb | k) ? 1u : 0u);
+                            umma_bf16(tmem_cross, a_lo + adv, b_hi + adv, idesc, 1u);
                         } else {
                             umma_bf16(tmem_main, a_hi + adv, b_hi + adv, idesc, acc_main);
                         }
@@ -216,10 +235,14 @@ k_syrk_tc(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CU
             }
             float* Hl = H + (size_t)(layer0 + l) * d * d;
             const int row = i0 + q * 32 + lane;
+            // split route: undo the power-of-two scales of the two feature rows (exact)
+            const unsigned* am = TF32 ? amax + (size_t)l * d : nullptr;
+            const float inv_row = (TF32 && row < d) ? row_scale(am[row], true) : 1.f;
 #pragma unroll
             for (int e = 0; e < NC; ++e) {
                 const int col = j0 + half * NC + e;
                 float val = alpha * (tot[e] + acc[e]);
+                if (TF32 && col < d) val = (val * inv_row) * row_scale(am[col], true);
                 if (row < d && col < d && col <= row) {
                     if (beta != 0.f) val += Hl[(size_t)row * d + col];
                     Hl[(size_t)row * d + col] = val;
@@ -257,10 +280,54 @@ __global__ void k_hessian_flag_timeout(float* __restrict__ H, int L, int d, cons
     if (l < L && *err_word != 0) H[(size_t)l * d * d] = __int_as_float(0x7fc00000);
 }
 
-// X_hi = X with the 13 low mantissa bits cleared (exactly a TF32 value), X_lo = X - X_hi (exact).
-__global__ void __launch_bounds__(256) k_split_tf32(const float* __restrict__ X, long long ldx,
-                                                    long long N, long long np, size_t rows,
-                                                    float* __restrict__ hi, float* __restrict__ lo) {
+// Largest magnitude of every feature row of a token-contiguous X (bit pattern of |x|, which
+// orders like the value for non-negative floats; a NaN sorts above everything and switches the
+// scaling of its row off).
+__global__ void __launch_bounds__(256) k_row_absmax(const float* __restrict__ X, long long ldx, long long N,
+                                                    unsigned* __restrict__ amax) {
+    __shared__ unsigned red[8];
+    const size_t row = blockIdx.x;
+    const float* src = X + row * (size_t)ldx;
+    unsigned m = 0u;
+    for (long long k = threadIdx.x; k < N; k += 256) m = max(m, __float_as_uint(src[k]) & 0x7fffffffu);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) m = max(m, red[w]);
+        amax[row] = m;
+    }
+}
+
+// The same for token-major input A [layers, N, lda] (one token per row): every thread walks one
+// feature over a slab of tokens, the slabs meet through atomicMax (amax zeroed beforehand).
+__global__ void __launch_bounds__(256) k_tokens_absmax(const float* __restrict__ A, long long lda,
+                                                       long long N, int d, long long slab,
+                                                       unsigned* __restrict__ amax) {
+    const int l = blockIdx.z;
+    const int f = blockIdx.x * 256 + threadIdx.x;
+    if (f >= d) return;
+    const long long t0 = (long long)blockIdx.y * slab, t1 = min(N, t0 + slab);
+    const float* Al = A + (size_t)l * (size_t)N * (size_t)lda + f;
+    unsigned m = 0u;
+    for (long long t = t0; t < t1; ++t) m = max(m, __float_as_uint(Al[(size_t)t * (size_t)lda]) & 0x7fffffffu);
+    atomicMax(amax + (size_t)l * d + f, m);
+}
+
+// The two fp16 parts of a scaled fp32 value y: y_1 = fp16(y), y_2 = fp16(y - y_1) (the difference
+// is exact in fp32).
+__device__ __forceinline__ void split_f16x2(float y, __half& p1, __half& p2) {
+    p1 = __float2half_rn(y);
+    p2 = __float2half_rn(y - __half2float(p1));
+}
+
+// X_1, X_2 of a token-contiguous fp32 X, four tokens per thread; np (a multiple of 8) is the row
+// pitch of the parts, zero past N.
+__global__ void __launch_bounds__(256) k_split_f16(const float* __restrict__ X, long long ldx,
+                                                   long long N, long long np, size_t rows,
+                                                   const unsigned* __restrict__ amax,
+                                                   __half* __restrict__ hi, __half* __restrict__ lo) {
     const size_t row = blockIdx.y;
     const long long k = ((long long)blockIdx.x * 256 + threadIdx.x) * 4;
     if (row >= rows || k >= np) return;
@@ -272,26 +339,26 @@ __global__ void __launch_bounds__(256) k_split_tf32(const float* __restrict__ X,
     } else {
         for (int e = 0; e < 4; ++e) if (k + e < N) v[e] = src[e];
     }
-    float h[4], w[4];
+    const float sc = row_scale(amax[row], false);
+    union { uint2 u; __half h[4]; } a, b;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        h[e] = __uint_as_float(__float_as_uint(v[e]) & 0xffffe000u);
-        w[e] = v[e] - h[e];
-    }
-    *reinterpret_cast<float4*>(hi + row * (size_t)np + k) = make_float4(h[0], h[1], h[2], h[3]);
-    *reinterpret_cast<float4*>(lo + row * (size_t)np + k) = make_float4(w[0], w[1], w[2], w[3]);
+    for (int e = 0; e < 4; ++e) split_f16x2(v[e] * sc, a.h[e], b.h[e]);
+    *reinterpret_cast<uint2*>(hi + row * (size_t)np + k) = a.u;
+    *reinterpret_cast<uint2*>(lo + row * (size_t)np + k) = b.u;
 }
 
 // Token-major input (one calibration token per row, as a forward pass emits activations):
 // A is [layers, N, lda] with the feature index contiguous.  A 32 x 32 tile goes through shared
 // memory, so the reads run along features and the writes along tokens, both coalesced; the output
-// is the K-major [layers * d, np] matrix the product kernel loads.  SPLIT writes the TF32 parts
-// X_hi / X_lo of an fp32 input directly (same values as k_split_tf32); otherwise the elements
-// are moved as raw bits (T = uint16_t for bf16).
-template <typename T, bool SPLIT>
+// is the K-major [layers * d, np] matrix the product kernel loads.  SPLIT writes the scaled fp16
+// parts X_1 / X_2 of an fp32 input directly (same values as k_split_f16; O = __half, amax holds
+// the features' largest magnitudes); otherwise the elements are moved as raw bits (T = O =
+// uint16_t for bf16 and fp16).
+template <typename T, typename O, bool SPLIT>
 __global__ void __launch_bounds__(256) k_tokens_to_kmajor(const T* __restrict__ A, long long lda,
                                                           long long N, int d, long long np,
-                                                          T* __restrict__ hi, T* __restrict__ lo) {
+                                                          const unsigned* __restrict__ amax,
+                                                          O* __restrict__ hi, O* __restrict__ lo) {
     __shared__ T tile[32][33];
     const int l = blockIdx.z;
     const long long t0 = (long long)blockIdx.x * 32;
@@ -313,9 +380,7 @@ __global__ void __launch_bounds__(256) k_tokens_to_kmajor(const T* __restrict__ 
         const size_t o = ((size_t)l * d + f) * (size_t)np + (size_t)t;
         const T v = tile[tx][r];
         if constexpr (SPLIT) {
-            const float h = __uint_as_float(__float_as_uint(v) & 0xffffe000u);
-            hi[o] = h;
-            lo[o] = v - h;
+            split_f16x2(v * row_scale(amax[(size_t)l * d + f], false), hi[o], lo[o]);
         } else {
             hi[o] = v;
         }
@@ -326,10 +391,11 @@ __global__ void __launch_bounds__(256) k_tokens_to_kmajor(const T* __restrict__ 
 // lda % 4 == 0): a 64 x 64 tile, four elements per access on both sides, so a row of the output
 // leaves in 256-byte (fp32) pieces.  np is a multiple of 4, so a quad that starts below np ends
 // below it.
-template <typename T, typename V, bool SPLIT>
+template <typename T, typename V, typename O, bool SPLIT>
 __global__ void __launch_bounds__(256) k_tokens_to_kmajor_v4(const T* __restrict__ A, long long lda,
                                                              long long N, int d, long long np,
-                                                             T* __restrict__ hi, T* __restrict__ lo) {
+                                                             const unsigned* __restrict__ amax,
+                                                             O* __restrict__ hi, O* __restrict__ lo) {
     __shared__ T tile[64][65];                       // [token][feature]
     union Quad { V v; T e[4]; };
     const int l = blockIdx.z;
@@ -365,14 +431,12 @@ __global__ void __launch_bounds__(256) k_tokens_to_kmajor_v4(const T* __restrict
         for (int e = 0; e < 4; ++e) u.e[e] = tile[4 * q + e][fl];
         const size_t o = ((size_t)l * d + f) * (size_t)np + (size_t)t;
         if constexpr (SPLIT) {
-            Quad h, w;
+            union { uint2 v; __half e[4]; } h, w;
+            const float sc = row_scale(amax[(size_t)l * d + f], false);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                h.e[e] = __uint_as_float(__float_as_uint(u.e[e]) & 0xffffe000u);
-                w.e[e] = u.e[e] - h.e[e];
-            }
-            *reinterpret_cast<V*>(hi + o) = h.v;
-            *reinterpret_cast<V*>(lo + o) = w.v;
+            for (int e = 0; e < 4; ++e) split_f16x2(u.e[e] * sc, h.e[e], w.e[e]);
+            *reinterpret_cast<uint2*>(hi + o) = h.v;
+            *reinterpret_cast<uint2*>(lo + o) = w.v;
         } else {
             *reinterpret_cast<V*>(hi + o) = u.v;
         }
@@ -418,7 +482,7 @@ int transpose_chunk_layers(int L, int d, long long N) {
 }
 
 int split_chunk_layers(int L, int d, long long N) {
-    const size_t per_layer = 2 * (size_t)d * (size_t)padded_tokens(N) * 4;
+    const size_t per_layer = 2 * (size_t)d * (size_t)padded_tokens_bf16(N) * 2;
     size_t lc = kSplitCapBytes / (per_layer ? per_layer : 1);
     if (lc < 1) lc = 1;
     return (int)(lc < (size_t)L ? lc : (size_t)L);
@@ -430,7 +494,8 @@ size_t hessian_tc_workspace_bytes(int L, int d, long long N, ziplm_dtype dt, boo
     size_t b = kAlign;   // error word
     if (dt == ZIPLM_F32) {
         const int lc = split_chunk_layers(L, d, N);
-        b += 2 * align_up((size_t)lc * d * (size_t)padded_tokens(N) * 4);
+        b += align_up((size_t)lc * d * sizeof(unsigned));                            // row magnitudes
+        b += 2 * align_up((size_t)lc * d * (size_t)padded_tokens_bf16(N) * 2);       // the two fp16 parts
     } else if (token_major) {
         const int lc = transpose_chunk_layers(L, d, N);
         b += align_up((size_t)lc * d * (size_t)padded_tokens_bf16(N) * 2);
@@ -461,46 +526,59 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
                                               (int)smem_bf16));
     }
     if (f32) {
-        const long long np = padded_tokens(N);
+        const long long np = padded_tokens_bf16(N);
         const int lc = split_chunk_layers(L, d, N);
-        float* hi = c.take<float>((size_t)lc * d * np);
-        float* lo = c.take<float>((size_t)lc * d * np);
+        unsigned* amax = c.take<unsigned>((size_t)lc * d);
+        __half* hi = c.take<__half>((size_t)lc * d * np);
+        __half* lo = c.take<__half>((size_t)lc * d * np);
         const int num_kb = (int)((N + Cfg<true>::BK - 1) / Cfg<true>::BK);
         for (int l0 = 0; l0 < L; l0 += lc) {
             const int ln = (L - l0 < lc) ? (L - l0) : lc;
             const size_t rows = (size_t)ln * d;
             if (token_major) {
                 const float* Ac = static_cast<const float*>(X) + (size_t)l0 * (size_t)N * ldx;
+                ZIPLM_CHECK_CUDA(cudaMemsetAsync(amax, 0, sizeof(unsigned) * rows, st));
+                // slabs of at least 256 tokens, at most 65535 of them (grid.y)
+                const long long slab = N / 65535 + 1 > 256 ? N / 65535 + 1 : 256;
                 // grid.z is limited to 65535 layers per launch
                 for (int z0 = 0; z0 < ln; z0 += 65535) {
                     const int zn = ln - z0 < 65535 ? ln - z0 : 65535;
+                    k_tokens_absmax<<<dim3((unsigned)((d + 255) / 256), (unsigned)((N + slab - 1) / slab),
+                                           (unsigned)zn), 256, 0, st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, slab,
+                                                                        amax + (size_t)z0 * d);
+                    ZIPLM_CHECK_LAUNCH();
                     if (quad_rows(X, ldx, 4))
-                        k_tokens_to_kmajor_v4<float, float4, true>
+                        k_tokens_to_kmajor_v4<float, float4, __half, true>
                             <<<dim3((unsigned)((np + 63) / 64), (unsigned)((d + 63) / 64), (unsigned)zn), 256,
-                               0, st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, np, hi + (size_t)z0 * d * np,
-                                        lo + (size_t)z0 * d * np);
+                               0, st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, np, amax + (size_t)z0 * d,
+                                        hi + (size_t)z0 * d * np, lo + (size_t)z0 * d * np);
                     else
-                        k_tokens_to_kmajor<float, true>
+                        k_tokens_to_kmajor<float, __half, true>
                             <<<dim3((unsigned)((np + 31) / 32), (unsigned)((d + 31) / 32), (unsigned)zn), 256,
-                               0, st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, np, hi + (size_t)z0 * d * np,
-                                        lo + (size_t)z0 * d * np);
+                               0, st>>>(Ac + (size_t)z0 * N * ldx, ldx, N, d, np, amax + (size_t)z0 * d,
+                                        hi + (size_t)z0 * d * np, lo + (size_t)z0 * d * np);
                     ZIPLM_CHECK_LAUNCH();
                 }
             } else {
                 const float* Xc = static_cast<const float*>(X) + (size_t)l0 * d * ldx;
+                for (size_t r0 = 0; r0 < rows; r0 += (size_t)1 << 30) {
+                    const size_t rn = rows - r0 < ((size_t)1 << 30) ? rows - r0 : ((size_t)1 << 30);
+                    k_row_absmax<<<(unsigned)rn, 256, 0, st>>>(Xc + r0 * ldx, ldx, N, amax + r0);
+                    ZIPLM_CHECK_LAUNCH();
+                }
                 // grid.y is limited to 65535 rows per launch
                 for (size_t r0 = 0; r0 < rows; r0 += 65535) {
                     const size_t rn = rows - r0 < 65535 ? rows - r0 : 65535;
-                    k_split_tf32<<<dim3((unsigned)((np / 4 + 255) / 256), (unsigned)rn), 256, 0, st>>>(
-                        Xc + r0 * ldx, ldx, N, np, rn, hi + r0 * np, lo + r0 * np);
+                    k_split_f16<<<dim3((unsigned)((np / 4 + 255) / 256), (unsigned)rn), 256, 0, st>>>(
+                        Xc + r0 * ldx, ldx, N, np, rn, amax + r0, hi + r0 * np, lo + r0 * np);
                     ZIPLM_CHECK_LAUNCH();
                 }
             }
             CUtensorMap mh, ml;
-            if (!make_map(&mh, hi, ZIPLM_F32, N, d, ln, np) || !make_map(&ml, lo, ZIPLM_F32, N, d, ln, np))
+            if (!make_map(&mh, hi, ZIPLM_F16, N, d, ln, np) || !make_map(&ml, lo, ZIPLM_F16, N, d, ln, np))
                 return ZIPLM_ERR_CUDA;
             k_syrk_tc<true><<<dim3(n_tiles, ln), THREADS, smem_tf32, st>>>(mh, ml, H, d, num_kb, alpha, beta,
-                                                                      l0, err_word, 2u, spin);
+                                                                      l0, err_word, 0u, spin, amax);
             ZIPLM_CHECK_LAUNCH();
         }
     } else if (token_major) {
@@ -513,18 +591,18 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
             const int ln = (L - l0 < lc) ? (L - l0) : lc;
             const uint16_t* Ac = static_cast<const uint16_t*>(X) + (size_t)l0 * (size_t)N * ldx;
             if (quad_rows(X, ldx, 2))
-                k_tokens_to_kmajor_v4<uint16_t, uint2, false>
+                k_tokens_to_kmajor_v4<uint16_t, uint2, uint16_t, false>
                     <<<dim3((unsigned)((np + 63) / 64), (unsigned)((d + 63) / 64), (unsigned)ln), 256, 0, st>>>(
-                        Ac, ldx, N, d, np, xt, nullptr);
+                        Ac, ldx, N, d, np, nullptr, xt, nullptr);
             else
-                k_tokens_to_kmajor<uint16_t, false>
+                k_tokens_to_kmajor<uint16_t, uint16_t, false>
                     <<<dim3((unsigned)((np + 31) / 32), (unsigned)((d + 31) / 32), (unsigned)ln), 256, 0, st>>>(
-                        Ac, ldx, N, d, np, xt, nullptr);
+                        Ac, ldx, N, d, np, nullptr, xt, nullptr);
             ZIPLM_CHECK_LAUNCH();
             CUtensorMap mx;
             if (!make_map(&mx, xt, dt, N, d, ln, np)) return ZIPLM_ERR_CUDA;
             k_syrk_tc<false><<<dim3(n_tiles, ln), THREADS, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
-                                                                       l0, err_word, fmt16, spin);
+                                                                       l0, err_word, fmt16, spin, nullptr);
             ZIPLM_CHECK_LAUNCH();
         }
     } else {
@@ -537,7 +615,7 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
             const __nv_bfloat16* Xc = static_cast<const __nv_bfloat16*>(X) + (size_t)l0 * d * ldx;
             if (!make_map(&mx, Xc, dt, N, d, ln, ldx)) return ZIPLM_ERR_CUDA;
             k_syrk_tc<false><<<dim3(n_tiles, ln), THREADS, smem_bf16, st>>>(mx, mx, H, d, num_kb, alpha, beta,
-                                                                       l0, err_word, fmt16, spin);
+                                                                       l0, err_word, fmt16, spin, nullptr);
             ZIPLM_CHECK_LAUNCH();
         }
     }
