@@ -600,7 +600,7 @@ def run_ours(args, shape):
         fma_peak = 35.7                                # fp32 TFMA/s measured with a register-only FMA loop
         hs_ms, _ = phases.get("hessian", (0.0, 0))
         hs_useful = float(L) * d * d * N                      # lower triangle: d^2 N flop per layer
-        tf32_peak = 1115.0    # TFLOP/s: tcgen05.mma kind::tf32, M = 128, N >= 128, operands in shared memory
+        f16_peak = 2225.0     # TFLOP/s: tcgen05.mma kind::f16, M = 128, N >= 128, operands in shared memory
         line = dict(
             metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
             warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
@@ -658,18 +658,21 @@ def run_ours(args, shape):
                                         "71.4 TFLOP/s fp32 (nominal 148 SMs x 128 lanes x 1.965 GHz "
                                         "= 74.4)")),
             roofline_hessian=dict(
-                kernel="k_split_tf32 + k_syrk_tc<tf32>", bound="tensor",
-                achieved=3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0, peak=tf32_peak,
-                unit="TFLOP/s", frac=(3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 / tf32_peak) if hs_ms > 0 else 0.0,
+                kernel="k_row_absmax + k_split_f16 + k_syrk_tc<split>", bound="tensor",
+                achieved=3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0, peak=f16_peak,
+                unit="TFLOP/s", frac=(3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 / f16_peak) if hs_ms > 0 else 0.0,
                 useful_tflops=hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0,
                 traffic=None, ms=hs_ms,
-                peak_source="measured on this part: one thread per SM issuing tcgen05.mma kind::tf32 "
-                            "128 x 128 x 8 back to back from shared-memory operands, 1114 TFLOP/s at "
-                            "N = 128 and 1116 at N = 256 (735 at N = 64; kind::f16 bf16 the same way: "
-                            "2225); nominal 1.1 PFLOP/s",
-                note="fp32 activations: every product is three TF32 MMAs (hi*hi, hi*lo, lo*hi), so "
-                     "the tensor-pipe work is 3 x the useful d^2 N flop per layer; the time is that "
-                     "of the whole call, the split pre-pass included"),
+                peak_source="measured on this part: one thread per SM issuing tcgen05.mma kind::f16 "
+                            "128 x 128 x 16 back to back from shared-memory operands, 2222 TFLOP/s at "
+                            "N = 128 and 2228 at N = 256 (1484 at N = 64; kind::tf32 the same way: "
+                            "1115); nominal 2.25 PFLOP/s",
+                note="fp32 activations: every feature row is scaled by a power of two and split "
+                     "into two fp16 parts, every product is three fp16 MMAs (x1*x1, x1*x2, x2*x1), "
+                     "so the tensor-pipe work is 3 x the useful d^2 N flop per layer; the time is "
+                     "that of the whole call, the row-maximum and split pre-passes included; the "
+                     "kernel is bound by its L2 -> shared-memory operand traffic (64 KB per K "
+                     "block of 64 tokens against 816 clocks of MMAs)"),
             roofline_streaming_update=dict(
                 kernel="k_neuron_update", bound="hbm", achieved=achieved, peak=peak, unit="GB/s",
                 frac=achieved / peak,

@@ -60,7 +60,8 @@ const char* ziplm_status_string(ziplm_status s);
  *
  * alpha = 2 gives the paper's Hessian; beta = 1 adds one more batch of tokens to a running sum,
  * beta = 0 overwrites.  Products are accumulated in fp32; fp32 inputs keep fp32 accuracy (on the
- * tensor-core route they are split into TF32 terms), bf16 and fp16 inputs are multiplied exactly
+ * tensor-core route every feature row is scaled by a power of two and split into two fp16 parts,
+ * three exact partial products per product, about 21 significant bits), bf16 and fp16 inputs are multiplied exactly
  * (an fp16 or bf16 product has at most 22 significant bits).
  *
  *   H          dev, [L, d, d] fp32, in/out; full symmetric matrix on return
@@ -97,7 +98,7 @@ ziplm_status ziplm_hessian_accumulate(float* H, const void* X, ziplm_dtype x_dty
  * X[l].  Calling it once per calibration batch with beta = 1 (beta = 0 on the first batch, or on a
  * zeroed H) builds the Hessian of the whole calibration set without ever holding all activations.
  * Arithmetic and accuracy are those of ziplm_hessian_accumulate: a pre-pass brings the batch into
- * the token-contiguous layout (for fp32 together with the TF32 split) and the same tensor-core
+ * the token-contiguous layout (for fp32 together with the fp16 split) and the same tensor-core
  * product kernel runs on it.
  *
  *   H          dev, [L, d, d] fp32, in/out; full symmetric matrix on return
