@@ -168,14 +168,18 @@ class ClockSampler:
 # CUDA leg
 # ------------------------------------------------------------------------------------------
 LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in prune_lazy.cu)
+LAZY_REFRESH = 64 # survivors at which that path rebuilds its state exactly (kRefresh there)
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch: constants from earlier
 # ncu captures of these kernels (taken on 4 of the 12 layers and scaled by 3: traffic grows in
 # proportion to the layers), not measurements of this run.  Only valid for the bench workload.
 NCU_TRAFFIC = {
-    # k_lazy_update_aq, first block at full size (12 layers, n_new = 3040)
-    "k_lazy_update_aq": dict(bytes=523.1e6 + 826.2e6, launch="n_new = 3040, m = 32, 12 layers",
-                             algorithmic=12 * 24.0 * 3040 * 3039 / 2),
+    # k_lazy_update_aq_tc, first block at full size (12 layers, 3072 positions of which 3040 live)
+    "k_lazy_update_aq_tc": dict(bytes=3 * (166.8e6 + 249.1e6), launch="n_pos = 3072, m = 32, 12 layers",
+                                algorithmic=12 * 24.0 * 3040 * 3039 / 2),
+    # k_lazy_update_aq, a compaction block near full size (12 layers, n_new = 2944)
+    "k_lazy_update_aq": dict(bytes=3 * (162.5e6 + 217.5e6), launch="n_new = 2944, m = 32, 12 layers",
+                             algorithmic=12 * 24.0 * 2944 * 2943 / 2),
     # k_dgemm_tiles, top-level product F21 = A21 M11^T
     "k_dgemm_tiles": dict(bytes=3 * (116.6e6 + 49.0e6), launch="F21 = A21 M11^T, 12 x 24 macro tiles",
                           algorithmic=None),
@@ -186,10 +190,12 @@ NCU_TRAFFIC = {
 
 
 def lazy_update_work(L, G, levels):
-    """Algorithmic work of k_lazy_update_aq over one greedy run: a launch that leaves n live
-    structures reads the off-diagonal entries of H^-1 and Q once per symmetric pair and writes
-    them at [i][j] and [j][i] (2 matrices x n(n-1)/2 pairs x 4 B x (1 read + 2 writes)) and spends
-    3 fp32 FMA per pair and pending step.
+    """Algorithmic work of the rank-32 update of H^-1 and Q (k_lazy_update_aq_tc in blocks that
+    leave removed positions in place, k_lazy_update_aq in blocks that squeeze them out) over one
+    greedy run: a launch that leaves n live structures reads the off-diagonal entries of H^-1 and
+    Q once per symmetric pair and writes them at [i][j] and [j][i] (2 matrices x n(n-1)/2 pairs x
+    4 B x (1 read + 2 writes)) and spends 3 fp32 FMA per pair and pending step.  Rows and columns
+    of removed positions that a dense block still carries are overhead, not counted here.
     Block boundaries fall on the requested levels, as in the library.  Returns (bytes, fma,
     launches)."""
     n, slot, nbytes, fma, launches = G, 0, 0.0, 0.0, 0
@@ -197,6 +203,8 @@ def lazy_update_work(L, G, levels):
     n_min = levels[-1] if levels else G
     while n > n_min:
         stop = levels[slot] if slot < len(levels) else n_min
+        if n > LAZY_REFRESH and stop < LAZY_REFRESH:
+            stop = LAZY_REFRESH          # the exact rebuild of the state ends a block
         m = min(LAZY_BLOCK, n - stop)
         n -= m
         if n > 1:
@@ -224,6 +232,8 @@ def run_ours(args, shape):
 
     if args.layer_groups:
         z.set_option(z.Option.LAYER_GROUPS, args.layer_groups)
+    if args.compact_every_block:
+        z.set_option(z.Option.COMPACT_EVERY_BLOCK, 1)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -635,10 +645,13 @@ def run_ours(args, shape):
                                       "= 37.2)",
                           note="float64 tile products of the Cholesky factor and its inverse "
                                "(2/3 d^3 flop per layer)"),
-            roofline=dict(kernel="k_lazy_update_aq", bound="hbm", achieved=aq_gbs, peak=peak,
+            roofline=dict(kernel="k_lazy_update_aq_tc (dense blocks) + k_lazy_update_aq (compaction blocks)",
+                          bound="hbm", achieved=aq_gbs, peak=peak,
                           unit="GB/s", frac=aq_gbs / peak,
-                          traffic=NCU_TRAFFIC["k_lazy_update_aq"]["bytes"] if full_workload else None,
-                          traffic_note=NCU_TRAFFIC["k_lazy_update_aq"], peak_source=peak_src,
+                          traffic=NCU_TRAFFIC["k_lazy_update_aq_tc"]["bytes"] if full_workload else None,
+                          traffic_note=dict(dense=NCU_TRAFFIC["k_lazy_update_aq_tc"],
+                                            compaction=NCU_TRAFFIC["k_lazy_update_aq"]),
+                          peak_source=peak_src,
                           launches=aq_n, avg_launch_us=1e3 * aq_ms / max(aq_n, 1),
                           algorithmic_bytes_per_step=aq_bytes,
                           symmetric=dict(bytes_per_step=aq_bytes * 16.0 / 24.0,
@@ -647,11 +660,16 @@ def run_ours(args, shape):
                                               "symmetric matrices (16 B per pair); the kernel's own "
                                               "count (24 B) includes the second, mirrored store that "
                                               "lets the steps kernel read a pivot column as a row"),
-                          note="rank-32 update of H^-1 and Q, the kernel with the largest summed time "
-                               "in the timed path; bound by its 4-byte gather through the compaction "
-                               "map (a stand-alone kernel with the same gather, mirror and direct "
-                               "stores and no arithmetic reaches 3.3-3.9 TB/s on this part, 4.7 with "
-                               "16-byte aligned reads), with the fp32 issue rate close behind (see alu)",
+                          note="rank-32 update of H^-1 and Q, the operation with the largest summed "
+                               "time in the timed path (the phase also holds the small kernel that "
+                               "packs the pending vectors for the tensor cores).  About three blocks "
+                               "in four leave removed positions in place and run dense 128 x 128 "
+                               "tiles on tcgen05 (bf16 x 3 split of the rank-32 operands, TMA loads, "
+                               "direct and mirrored stores); the others squeeze removed positions "
+                               "out with 4-byte gathers on the CUDA cores.  A stand-alone kernel "
+                               "with this traffic shape (one read, a direct and a mirrored store per "
+                               "entry) and no arithmetic reaches 5.0-5.2 TB/s on this part, 3.3-3.9 "
+                               "TB/s with the gather in front",
                           alu=dict(achieved_tfma=aq_fma / (aq_ms * 1e-3) / 1e12 if aq_ms > 0 else 0.0,
                                    peak_tfma=fma_peak,
                                    note="3 fp32 FMA per entry and pending step; peak = measured "
@@ -722,6 +740,9 @@ def main():
                     help="profiling aid: use only this many of the workload's layers")
     ap.add_argument("--max-removed", type=int, default=0,
                     help="profiling aid: stop the greedy loop after this many removals")
+    ap.add_argument("--compact-every-block", action="store_true",
+                    help="delayed-update path: squeeze removed positions out after every block "
+                         "(the gathering CUDA-core update only; profiling aid)")
     ap.add_argument("--layer-groups", type=int, default=0,
                     help="profiling aid: number of layer groups on internal streams (0 = library default; "
                          "1 runs them back to back, so that a profiler's per-kernel times add up)")

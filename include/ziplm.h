@@ -367,6 +367,11 @@ ziplm_status ziplm_search_levels(const float* loss, const float* base_loss, cons
  *     ZIPLM_OPT_SPIN_LIMIT        0: default; n > 0: poll limit of the Hessian kernel's wait for a
  *                                 free pipeline stage (tests make a bounded wait run out with it;
  *                                 see ziplm_hessian_accumulate for how that is reported).
+ *     ZIPLM_OPT_COMPACT_EVERY_BLOCK  0: the delayed-update neuron path leaves removed positions in
+ *                                 place for a few blocks (dense tensor-core update of H^-1 and Q)
+ *                                 and squeezes them out when 128 of them, or a sixteenth of all
+ *                                 positions, have gathered; 1: squeezes them out after every
+ *                                 block (gathering CUDA-core update only).
  * ziplm_get_option         current value of an option.
  * ziplm_launch_count       kernels launched by this library since it was loaded.
  * ziplm_profile_begin      from now on every phase of every call is bracketed by a pair of CUDA
@@ -384,7 +389,8 @@ typedef enum {
     ZIPLM_OPT_FORCE_BLOCK_PATH = 2,
     ZIPLM_OPT_HESSIAN_ROUTE = 3,
     ZIPLM_OPT_SPIN_LIMIT = 4,
-    ZIPLM_OPT_COUNT = 5
+    ZIPLM_OPT_COMPACT_EVERY_BLOCK = 5,
+    ZIPLM_OPT_COUNT = 6
 } ziplm_option;
 ziplm_status ziplm_set_option(ziplm_option option, int value);
 int ziplm_get_option(ziplm_option option);

@@ -448,6 +448,7 @@ class Option:
     FORCE_BLOCK_PATH = 2     # 1: group_size 1 through the general block path
     HESSIAN_ROUTE = 3        # 1: CUDA-core Hessian kernel always
     SPIN_LIMIT = 4           # poll limit of the Hessian kernel's wait for a free pipeline stage
+    COMPACT_EVERY_BLOCK = 5  # 1: squeeze removed positions out after every block of the neuron path
 
 
 def set_option(option: int, value: int) -> None:

@@ -38,7 +38,7 @@ int option_value(int option);
 // Phases reported by the optional event timing (ziplm_profile_begin / ziplm_profile_end).
 enum Phase { PH_HESSIAN = 0, PH_INVERSE, PH_INIT, PH_PREP, PH_UPDATE, PH_SNAPSHOT, PH_BLOCK_SCORE,
              PH_BLOCK_UPDATE, PH_LAZY_STEPS, PH_LAZY_UPDATE_AQ, PH_LAZY_UPDATE_W, PH_INV_PRODUCTS,
-             PH_INV_LEAVES, PH_INV_LAUUM, PH_COUNT };
+             PH_INV_LEAVES, PH_INV_LAUUM, PH_LAZY_REFRESH, PH_COUNT };
 
 // Brackets the launches issued during its lifetime with a pair of events when timing is on.
 struct PhaseScope {

@@ -25,7 +25,7 @@ std::vector<Span> g_spans;
 const char* kPhaseNames[PH_COUNT] = {"hessian", "inverse", "init", "prep", "update", "snapshot",
                                      "block_score", "block_update", "lazy_steps", "lazy_update_aq",
                                      "lazy_update_w", "inverse_products", "inverse_leaves",
-                                     "inverse_lauum"};
+                                     "inverse_lauum", "lazy_refresh"};
 }  // namespace
 
 PhaseScope::PhaseScope(int phase, cudaStream_t st) : st_(st), idx_(-1) {
@@ -57,7 +57,7 @@ long long ziplm_launch_count(void) { return g_launches.load(); }
 ziplm_status ziplm_set_option(ziplm_option option, int value) {
     if (option < 0 || option >= ZIPLM_OPT_COUNT || value < 0) return ZIPLM_ERR_INVALID_ARG;
     if ((option == ZIPLM_OPT_NEURON_PATH || option == ZIPLM_OPT_FORCE_BLOCK_PATH ||
-         option == ZIPLM_OPT_HESSIAN_ROUTE) && value > 1)
+         option == ZIPLM_OPT_HESSIAN_ROUTE || option == ZIPLM_OPT_COMPACT_EVERY_BLOCK) && value > 1)
         return ZIPLM_ERR_INVALID_ARG;
     if (option == ZIPLM_OPT_LAYER_GROUPS && value > 8) return ZIPLM_ERR_INVALID_ARG;
     ziplm::g_options[option].store(value, std::memory_order_relaxed);

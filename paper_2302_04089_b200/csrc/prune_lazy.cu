@@ -29,9 +29,21 @@
 #include <math.h>
 
 
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace ziplm {
+
+// Tensor-core rank-32 update of H^-1 and Q for blocks that leave every position in place
+// (prune_lazy_tc.cu).
+size_t lazy_tc_pack_floats(int L, int d);
+bool lazy_tc_make_map(CUtensorMap* m, const float* P, int L, int d);
+bool lazy_tc_make_matrix_map(CUtensorMap* m, const float* M, int L, int d);
+ziplm_status run_lazy_update_aq_tc(const CUtensorMap& map, const CUtensorMap& map_a,
+                                   const CUtensorMap& map_q, int L, int n_pos, int m, int d, float* A2,
+                                   float* Q2, const float* U, const float* Z, float* P, int* counter,
+                                   int* layer_status, unsigned slot_spin_limit, cudaStream_t st);
 
 namespace {
 
@@ -39,6 +51,8 @@ constexpr int BMAX = 32;         // pending steps per block
 constexpr int STEP_THREADS = 256; // threads per CTA of the steps kernel, four positions each
 constexpr int SLICE_MAX = 768;   // positions per CTA: 2 * BMAX * SLICE_MAX * 4 B = 192 KiB of smem
 constexpr int CLUSTER_MAX = 8;   // portable cluster size
+constexpr int kDeadMax = 128;    // removed positions tolerated in the arrays before they are squeezed out
+constexpr int kDeadFraction = 16; // ... or this fraction of all positions, whichever comes first
 
 struct LazyState {
     double sumrho;
@@ -171,7 +185,7 @@ __device__ __forceinline__ Cand warp_best(const Cand& mine) { return warp_best(m
 // of the block by forward substitution with the 32 x 32 triangle T[m][s] = u_s[p_m].
 // Finally the per-position vectors are compacted (stable) across the cluster.
 __global__ void __launch_bounds__(STEP_THREADS, 1)
-k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
+k_lazy_steps(int n0, int S, int t0, int nsteps, int compact, int d, int G, int r, int rp,
              const float* __restrict__ A, const float* __restrict__ Q, const float* __restrict__ Wt,
              const double* __restrict__ dA_in, const double* __restrict__ dQ_in,
              const int* __restrict__ idx_in, double* __restrict__ dA_out,
@@ -214,10 +228,13 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const int k = k0 + e;
-        alive[e] = owner_thread && k < n0;
+        // a position removed in an earlier block that has not been squeezed out yet carries
+        // index -1: it stays dead
+        const int o = (owner_thread && k < n0) ? idx_in[(size_t)l * d + k] : -1;
+        alive[e] = o >= 0;
         da[e] = alive[e] ? dA_in[(size_t)l * d + k] : 1.0;
         dq[e] = alive[e] ? dQ_in[(size_t)l * d + k] : 0.0;
-        org[e] = alive[e] ? idx_in[(size_t)l * d + k] : 0x7fffffff;
+        org[e] = alive[e] ? o : 0x7fffffff;
     }
     double sumrho = 0.0;                       // meaningful in thread 0 of rank 0
 
@@ -364,7 +381,28 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int d, int G, int r, int rp,
         }
     }
 
-    // ---- stable compaction of the per-position vectors across the cluster; src[new] = old
+    // ---- end of the block.  Either the removed positions are squeezed out (stable compaction of
+    //      the per-position vectors across the cluster; src[new] = old), or every position stays
+    //      where it is (src = identity) and the removed ones are marked with index -1: the update
+    //      kernels then move nothing and a later block does the squeezing.
+    if (!compact) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int k = k0 + e;
+            if (owner_thread && k < n0) {
+                src[(size_t)l * d + k] = k;
+                dA_out[(size_t)l * d + k] = da[e];
+                dQ_out[(size_t)l * d + k] = dq[e];
+                idx_out[(size_t)l * d + k] = alive[e] ? org[e] : -1;
+            }
+        }
+        if (rank == 0 && tid == 0) {
+            state[l].sumrho += sumrho;
+            state[l].n_new = n0;
+        }
+        cluster.sync();      // no CTA may retire while another can still read its shared memory
+        return;
+    }
     const int f0 = alive[0] ? 1 : 0, f1 = alive[1] ? 1 : 0, f2 = alive[2] ? 1 : 0, f3 = alive[3] ? 1 : 0;
     const int mine = f0 + f1 + f2 + f3;
     int incl = mine;
@@ -631,13 +669,135 @@ __global__ void __launch_bounds__(256, 3) k_lazy_update_w(int n_new, int m, int 
     }
 }
 
+// Exact refresh of the state of the last kRefresh structures.  By then the surviving entries of
+// H^-1 have been reduced by orders of magnitude through thousands of fp32 downdates, and the
+// relative error of the saliencies, below 5e-6 until about 64 structures remain, would grow to
+// 1e-4 over the last steps.  H^-1 restricted to the survivors is the inverse of H_lambda
+// restricted to them (Sec. 3.1, the remark on Eq. 4), and Q is the Gram matrix of the current
+// weight columns, so both are rebuilt here from their definitions in float64: one CTA per layer,
+// n <= 64 compacted positions; CTA (l, 0) does the Cholesky, the inverse of the factor and M^T M
+// in shared memory, CTA (l, 1) the Gram matrix.
+constexpr int kRefresh = 64;
+__device__ void lazy_refresh_gram(int n, int d, int r, int rp, const float* __restrict__ Wl,
+                                  float* __restrict__ Ql, double* __restrict__ dQl, float* sW);
+__global__ void __launch_bounds__(256) k_lazy_refresh(int n, int d, int r, int rp,
+                                                      const float* __restrict__ H,
+                                                      const double* __restrict__ lam,
+                                                      const int* __restrict__ idx,
+                                                      const float* __restrict__ Wt, float* __restrict__ A,
+                                                      float* __restrict__ Q, double* __restrict__ dA,
+                                                      double* __restrict__ dQ, int* layer_status) {
+    extern __shared__ double dyn_refresh[];
+    double (*sB)[kRefresh + 1] = reinterpret_cast<double (*)[kRefresh + 1]>(dyn_refresh);
+    double (*sI)[kRefresh + 1] = reinterpret_cast<double (*)[kRefresh + 1]>(dyn_refresh + kRefresh * (kRefresh + 1));
+    __shared__ int sidx[kRefresh];
+    __shared__ int flag;
+    const int l = blockIdx.x, tid = threadIdx.x;
+    if (blockIdx.y == 1) {
+        lazy_refresh_gram(n, d, r, rp, Wt + (size_t)l * d * rp, Q + (size_t)l * d * d,
+                          dQ + (size_t)l * d, reinterpret_cast<float*>(dyn_refresh));
+        return;
+    }
+    const float* Hl = H + (size_t)l * d * d;
+    float* Al = A + (size_t)l * d * d;
+    if (tid == 0) flag = 0;
+    if (tid < n) sidx[tid] = idx[(size_t)l * d + tid];
+    __syncthreads();
+    for (int e = tid; e < n * n; e += 256) {
+        const int i = e / n, j = e % n;
+        sB[i][j] = (double)Hl[(size_t)sidx[i] * d + sidx[j]] + (i == j ? lam[l] : 0.0);
+    }
+    __syncthreads();
+    // Cholesky B = C C^T, column by column
+    for (int c = 0; c < n; ++c) {
+        if (tid == 0) {
+            double p = sB[c][c];
+            if (!(p > 0.0) || !isfinite(p)) {
+                if (!flag) flag = isfinite(p) ? ZIPLM_ERR_NOT_PD : ZIPLM_ERR_NONFINITE;
+                p = 1.0;
+            }
+            sB[c][c] = sqrt(p);
+        }
+        __syncthreads();
+        for (int i = c + 1 + tid; i < n; i += 256) sB[i][c] /= sB[c][c];
+        __syncthreads();
+        const int m = n - 1 - c;
+        for (int e = tid; e < m * m; e += 256) {
+            const int i = c + 1 + e / m, jj = c + 1 + e % m;
+            if (jj <= i) sB[i][jj] -= sB[i][c] * sB[jj][c];
+        }
+        __syncthreads();
+    }
+    // M = C^-1, one thread per column
+    if (tid < n) {
+        const int j = tid;
+        for (int k = 0; k < j; ++k) sI[k][j] = 0.0;
+        for (int k = j; k < n; ++k) {
+            double v = (k == j) ? 1.0 : 0.0;
+            for (int m = j; m < k; ++m) v -= sB[k][m] * sI[m][j];
+            sI[k][j] = v / sB[k][k];
+        }
+    }
+    __syncthreads();
+    // H^-1 = M^T M: fp32 off-diagonal entries in both triangles, float64 diagonal
+    for (int e = tid; e < n * n; e += 256) {
+        const int i = e / n, j = e % n;
+        double t = 0.0;
+        for (int k = (i > j ? i : j); k < n; ++k) t = fma(sI[k][i], sI[k][j], t);
+        if (i == j) dA[(size_t)l * d + i] = t;
+        else Al[(size_t)i * d + j] = (float)t;
+    }
+    if (tid == 0 && flag) set_layer_status(layer_status, l, flag);
+}
+
+// Second half of the refresh, CTA (l, 1): Q = W^T W on the surviving columns (rows of Wt),
+// float64 sums of the fp32 weights.  Chunks of 32 weights per row go through shared memory; every
+// thread owns a 4 x 4 tile of the n x n result.
+__device__ void lazy_refresh_gram(int n, int d, int r, int rp, const float* __restrict__ Wl,
+                                  float* __restrict__ Ql, double* __restrict__ dQl, float* sW) {
+    const int tid = threadIdx.x, ti = tid >> 4, tj = tid & 15;
+    double acc[4][4] = {};
+    for (int k0 = 0; k0 < r; k0 += 32) {
+        for (int e = tid; e < kRefresh * 32; e += 256) {
+            const int row = e >> 5, k = e & 31;
+            sW[row * 33 + k] = (row < n && k0 + k < r) ? Wl[(size_t)row * rp + k0 + k] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int k = 0; k < 32; ++k) {
+            double a[4], b[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                a[x] = (double)sW[(ti + 16 * x) * 33 + k];
+                b[x] = (double)sW[(tj + 16 * x) * 33 + k];
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y) acc[x][y] = fma(a[x], b[y], acc[x][y]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+            const int i = ti + 16 * x, j = tj + 16 * y;
+            if (i >= n || j >= n) continue;
+            if (i == j) dQl[i] = acc[x][y];
+            else Ql[(size_t)i * d + j] = (float)acc[x][y];
+        }
+}
+
 __global__ void __launch_bounds__(256) k_lazy_pos_of(int n, int d, const int* __restrict__ idx,
                                                      int* __restrict__ pos_of) {
     const int l = blockIdx.x;
     for (int c = threadIdx.x; c < d; c += blockDim.x) pos_of[(size_t)l * d + c] = -1;
     __syncthreads();
-    for (int k = threadIdx.x; k < n; k += blockDim.x)
-        pos_of[(size_t)l * d + idx[(size_t)l * d + k]] = k;
+    for (int k = threadIdx.x; k < n; k += blockDim.x) {
+        const int o = idx[(size_t)l * d + k];
+        if (o >= 0) pos_of[(size_t)l * d + o] = k;      // -1: removed, not squeezed out yet
+    }
 }
 
 // W_snap = current weights in original column order, removed columns exactly zero; accumulates
@@ -730,6 +890,7 @@ struct LazyWs {
     float* A[2]; float* Q[2]; float* Wt[2];
     double* dA[2]; double* dQ[2]; int* idx[2];
     int* src; int* pos_of; float* U; float* Z; float* C;
+    float* P; int* sched;              // packed operands and work counter of the tensor-core update
     LazyState* state; double* lam; double* base_acc;
     void* aux; size_t aux_bytes;       // shared by the inverse and by the Gram-matrix product
     int rp; size_t total;
@@ -750,6 +911,8 @@ LazyWs carve_lazy(void* ws, int L, int r, int d) {
     w.U = c.take<float>((size_t)L * BMAX * d);
     w.Z = c.take<float>((size_t)L * BMAX * d);
     w.C = c.take<float>((size_t)L * BMAX * w.rp);
+    w.P = c.take<float>(lazy_tc_pack_floats(L, d));
+    w.sched = c.take<int>(2);
     w.state = c.take<LazyState>((size_t)L);
     w.lam = c.take<double>((size_t)L);
     w.base_acc = c.take<double>((size_t)L);
@@ -833,16 +996,37 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
         if (s != ZIPLM_OK) return s;
     }
     const int n_min = n_levels > 0 ? levels[n_levels - 1] : G;
+    // n = live structures, npos = positions of the arrays (live ones and those removed since the
+    // last block that squeezed the removed positions out)
+    int npos = G;
+    const bool every_block = option_value(ZIPLM_OPT_COMPACT_EVERY_BLOCK) == 1;
+    CUtensorMap map_p, map_a[2], map_q[2];
+    if (!lazy_tc_make_map(&map_p, w.P, L, d)) return ZIPLM_ERR_CUDA;
+    for (int b = 0; b < 2; ++b)
+        if (!lazy_tc_make_matrix_map(&map_a[b], w.A[b], L, d) || !lazy_tc_make_matrix_map(&map_q[b], w.Q[b], L, d))
+            return ZIPLM_ERR_CUDA;
+    ZIPLM_CHECK_CUDA(cudaMemsetAsync(w.sched, 0, sizeof(int) * 2, st));
+    constexpr size_t kRefreshSmem = sizeof(double) * 2 * kRefresh * (kRefresh + 1);
+    ZIPLM_CHECK_CUDA(cudaFuncSetAttribute(k_lazy_refresh, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)kRefreshSmem));
     while (n > n_min) {
-        const int stop = (slot < n_levels) ? levels[slot] : n_min;   // next block boundary
+        int stop = (slot < n_levels) ? levels[slot] : n_min;         // next block boundary
+        if (n > kRefresh && stop < kRefresh) stop = kRefresh;        // ... and the refresh point
         const int nsteps = (n - stop < BMAX) ? (n - stop) : BMAX;
         const int nxt = cur ^ 1;
+        // Squeezing removed positions out makes the update kernels gather through a map; leaving
+        // them in place keeps their reads and writes dense at the price of dead rows and columns.
+        // They are squeezed out once they make up kDeadMax positions or a sixteenth of all.
+        const int dead_after = npos - (n - nsteps);
+        const bool refresh = (n > kRefresh && n - nsteps == kRefresh);
+        const int compact = (every_block || refresh || dead_after >= kDeadMax ||
+                             dead_after * kDeadFraction >= npos) ? 1 : 0;
         {
             PhaseScope ps(PH_LAZY_STEPS, st);
             // smallest cluster whose per-CTA slice of positions fits shared memory
             int cs = 1;
-            while (cs < CLUSTER_MAX && round_up_int((n + cs - 1) / cs, 4) > SLICE_MAX) cs *= 2;
-            const int S = round_up_int((n + cs - 1) / cs, 4);
+            while (cs < CLUSTER_MAX && round_up_int((npos + cs - 1) / cs, 4) > SLICE_MAX) cs *= 2;
+            const int S = round_up_int((npos + cs - 1) / cs, 4);
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(L * cs);
             cfg.blockDim = dim3(STEP_THREADS);
@@ -861,13 +1045,13 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
             cfg.attrs = attr;
             cfg.numAttrs = 2;
             ZIPLM_CHECK_CUDA(cudaLaunchKernelEx(
-                &cfg, k_lazy_steps, n, S, t, nsteps, d, G, r, rp, (const float*)w.A[cur],
+                &cfg, k_lazy_steps, npos, S, t, nsteps, compact, d, G, r, rp, (const float*)w.A[cur],
                 (const float*)w.Q[cur], (const float*)w.Wt[cur], (const double*)w.dA[cur],
                 (const double*)w.dQ[cur], (const int*)w.idx[cur], w.dA[nxt], w.dQ[nxt], w.idx[nxt],
                 w.src, w.U, w.Z, w.C, w.state, order, saliency, layer_status));
             ZIPLM_CHECK_LAUNCH();
         }
-        const int n_new = n - nsteps;
+        const int n_new = compact ? n - nsteps : npos;      // positions after this block
         // The update of W goes first: measured, the step is 2 ms shorter than with the wide update
         // of H^-1 and Q in front (the next steps kernel then follows the kernel with the longer,
         // finer-grained tail).
@@ -877,7 +1061,13 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
                 n_new, nsteps, d, rp, w.Wt[cur], w.Wt[nxt], w.src, w.U, w.C);
             ZIPLM_CHECK_LAUNCH();
         }
-        if (n_new > 1) {
+        if (n_new > 1 && !compact) {
+            // every position stays in place: dense tiles, tensor-core kernel
+            PhaseScope ps(PH_LAZY_UPDATE_AQ, st);
+            s = run_lazy_update_aq_tc(map_p, map_a[cur], map_q[cur], L, n_new, nsteps, d, w.A[nxt], w.Q[nxt],
+                                      w.U, w.Z, w.P, w.sched, layer_status, 0u, st);
+            if (s != ZIPLM_OK) return s;
+        } else if (n_new > 1) {
             PhaseScope ps(PH_LAZY_UPDATE_AQ, st);
             const int T = (n_new + 63) / 64;
             k_lazy_update_aq<<<dim3(T * (T + 1) / 2, L), 128, 0, st>>>(
@@ -885,10 +1075,18 @@ ziplm_status run_prune_lazy(const float* W, const float* H, int L, int r, int d,
             ZIPLM_CHECK_LAUNCH();
         }
         cur = nxt;
-        n = n_new;
+        npos = n_new;
+        n -= nsteps;
         t += nsteps;
+        if (refresh) {
+            PhaseScope ps(PH_LAZY_REFRESH, st);
+            k_lazy_refresh<<<dim3(L, 2), 256, kRefreshSmem, st>>>(npos, d, r, rp, H, w.lam, w.idx[cur],
+                                                                  w.Wt[cur], w.A[cur], w.Q[cur], w.dA[cur],
+                                                                  w.dQ[cur], layer_status);
+            ZIPLM_CHECK_LAUNCH();
+        }
         if (slot < n_levels && levels[slot] == n) {
-            s = snapshot(n, slot++);
+            s = snapshot(npos, slot++);
             if (s != ZIPLM_OK) return s;
         }
     }

@@ -58,12 +58,12 @@ def test_status_strings_and_workspace_queries(lib):
 def test_options_round_trip_and_reject_bad_values(lib):
     lib.ziplm_set_option.restype = ctypes.c_int
     lib.ziplm_get_option.restype = ctypes.c_int
-    for opt, good, bad in ((0, 1, 2), (1, 8, 9), (2, 1, 2), (3, 1, 5), (4, 1000, -1)):
+    for opt, good, bad in ((0, 1, 2), (1, 8, 9), (2, 1, 2), (3, 1, 5), (4, 1000, -1), (5, 1, 2)):
         assert lib.ziplm_get_option(opt) == 0
         assert lib.ziplm_set_option(opt, good) == 0 and lib.ziplm_get_option(opt) == good
         assert lib.ziplm_set_option(opt, bad) == 1 and lib.ziplm_get_option(opt) == good
         assert lib.ziplm_set_option(opt, 0) == 0
-    assert lib.ziplm_set_option(5, 0) == 1 and lib.ziplm_set_option(-1, 0) == 1
+    assert lib.ziplm_set_option(6, 0) == 1 and lib.ziplm_set_option(-1, 0) == 1
     assert lib.ziplm_get_option(17) == 0
 
 

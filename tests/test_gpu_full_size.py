@@ -59,9 +59,10 @@ def neuron_variant():
 
     def choose(path):
         z.set_option(z.Option.NEURON_PATH, 1 if path == "stream" else 0)
+        z.set_option(z.Option.COMPACT_EVERY_BLOCK, 1 if path == "lazy_compact" else 0)
 
     yield choose
-    z.set_option(z.Option.NEURON_PATH, 0)
+    choose("lazy")
 
 
 def generic_properties(shape, out):
@@ -138,7 +139,7 @@ def lockstep_head(W, H32, shape, out, layer, n_steps):
     return near
 
 
-@pytest.mark.parametrize("path", ["lazy", "stream"])
+@pytest.mark.parametrize("path", ["lazy", "lazy_compact", "stream"])
 def test_c3_bert_base_fc2_full_size_twelve_layers(path, neuron_variant):
     neuron_variant(path)
     shape = wl.CONFIGS["c3_bert_base_fc2"][0]

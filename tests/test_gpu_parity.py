@@ -222,14 +222,21 @@ def test_not_positive_definite_layer_is_flagged_and_others_finish():
 
 
 # ------------------------------------------------------------------ neuron path (a4 - a10)
-@pytest.fixture(params=["lazy", "stream"])
+def choose_neuron_path(z, name):
+    z.set_option(z.Option.NEURON_PATH, 1 if name == "stream" else 0)
+    z.set_option(z.Option.COMPACT_EVERY_BLOCK, 1 if name == "lazy_compact" else 0)
+
+
+@pytest.fixture(params=["lazy", "lazy_compact", "stream"])
 def neuron_path(request):
     """Run a test once per neuron-path variant: delayed rank-B updates (default where the shape
-    allows it) and the per-step streaming update."""
+    allows it; removed positions left in place between compactions, dense tensor-core update),
+    the same with a compaction after every block (gathering FMA update only), and the per-step
+    streaming update."""
     z = zb()
-    z.set_option(z.Option.NEURON_PATH, 1 if request.param == "stream" else 0)
+    choose_neuron_path(z, request.param)
     yield request.param
-    z.set_option(z.Option.NEURON_PATH, 0)
+    choose_neuron_path(z, "lazy")
 
 
 def test_c1_tiny_ffn_full_config(neuron_path):
@@ -259,14 +266,23 @@ def test_neuron_path_mid_size_full_depth_three_layers(neuron_path):
     print(reports)
 
 
-@pytest.mark.parametrize("d,check", [(1536, [0, 1]), (2048, [1])])
-def test_clustered_steps_kernel_full_depth_every_step(d, check):
+@pytest.mark.parametrize("d,check,variant", [(1536, [0, 1], "lazy"), (1536, [1], "lazy_compact"),
+                                             (2048, [1], "lazy")])
+def test_clustered_steps_kernel_full_depth_every_step(d, check, variant):
     """Full greedy order d -> 0 of the default path in lock-step with the oracle at widths where
     the steps kernel runs on clusters of 2 (769..1536 live positions) and 4 (1537..2048) CTAs, and
-    on one CTA from 768 down: every single pick is compared, and every level's snapshot and loss."""
+    on one CTA from 768 down: every single pick is compared, and every level's snapshot and loss.
+    Both update routes of the default path are covered (dense blocks on the tensor cores with
+    occasional compaction, and compaction after every block), and the exact rebuild of the state
+    at 64 survivors lies inside the compared range."""
+    z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=d, d_row=256, d_latent=d // 4,
                    n_tokens=2 * d, n_layers=2, levels=tuple(range(d - d // 8, -1, -d // 8)))
-    out, reports = run_case(sh, check_layers=check)
+    choose_neuron_path(z, variant)
+    try:
+        out, reports = run_case(sh, check_layers=check)
+    finally:
+        choose_neuron_path(z, "lazy")
     for rep in reports:
         assert rep["steps"] == d
     print(reports)
