@@ -206,6 +206,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int compact, int d, int G, int r
     float* sZ = sU + (size_t)BMAX * S;                     // [BMAX][S]
     __shared__ Cand s_cand[2][CLUSTER_MAX * NW];           // all warps of the cluster, by step parity
     __shared__ float sT[BMAX][BMAX];                       // T[m][s] = u_s[p_m]
+    __shared__ double sTd[BMAX][BMAX];                     // ... in float64, for the solve of c_m
     __shared__ float sUp[BMAX], sZp[BMAX];
     __shared__ int s_pm[BMAX];
     __shared__ double s_rsm[BMAX];
@@ -361,11 +362,17 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int compact, int d, int G, int r
     cluster.sync();
 
     // ---- c_m = (W[:,p_m] - sum_{s<m} c_s T[m][s]) / sqrt(h_m): forward substitution per row
-    //      index i of W, each CTA takes a slice of the d_row indices
-    {
+    //      index i of W, each CTA takes a slice of the d_row indices.  The triangle is widened to
+    //      float64 once, so that the inner loop is loads and FMAs only.  The solve reads this
+    //      CTA's own shared memory only and runs last, when the per-position state is dead.
+    auto solve_c = [&]() {
+        for (int e = tid; e < BMAX * BMAX; e += STEP_THREADS)
+            sTd[e / BMAX][e % BMAX] = (double)sT[e / BMAX][e % BMAX];
+        __syncthreads();
         const int per = (rp + CS - 1) / CS;
         for (int i = rank * per + tid; i < min(rp, (rank + 1) * per); i += STEP_THREADS) {
-            float w[BMAX], c[BMAX];
+            float w[BMAX];
+            double c[BMAX];          // the fp32 values that are stored, widened
 #pragma unroll
             for (int m = 0; m < BMAX; ++m)
                 w[m] = (m < nsteps && i < r) ? Wl[(size_t)s_pm[m] * rp + i] : 0.f;
@@ -373,13 +380,14 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int compact, int d, int G, int r
             for (int m = 0; m < BMAX; ++m) {
                 double acc[4] = {(double)w[m], 0.0, 0.0, 0.0};
 #pragma unroll
-                for (int s = 0; s < m; ++s)
-                    acc[s & 3] = fma(-(double)c[s], (double)sT[m][s], acc[s & 3]);
-                c[m] = (m < nsteps) ? (float)(((acc[0] + acc[1]) + (acc[2] + acc[3])) * s_rsm[m]) : 0.f;
-                if (m < nsteps) Cl[(size_t)m * rp + i] = c[m];
+                for (int s = 0; s < m; ++s) acc[s & 3] = fma(-c[s], sTd[m][s], acc[s & 3]);
+                const float cm =
+                    (m < nsteps) ? (float)(((acc[0] + acc[1]) + (acc[2] + acc[3])) * s_rsm[m]) : 0.f;
+                c[m] = (double)cm;
+                if (m < nsteps) Cl[(size_t)m * rp + i] = cm;
             }
         }
-    }
+    };
 
     // ---- end of the block.  Either the removed positions are squeezed out (stable compaction of
     //      the per-position vectors across the cluster; src[new] = old), or every position stays
@@ -401,6 +409,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int compact, int d, int G, int r
             state[l].n_new = n0;
         }
         cluster.sync();      // no CTA may retire while another can still read its shared memory
+        solve_c();
         return;
     }
     const int f0 = alive[0] ? 1 : 0, f1 = alive[1] ? 1 : 0, f2 = alive[2] ? 1 : 0, f3 = alive[3] ? 1 : 0;
@@ -435,6 +444,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int compact, int d, int G, int r
     if (rank == 0 && tid == 0) state[l].sumrho += sumrho;
     if (rank == CS - 1 && tid == 0) state[l].n_new = base + s_count;
     cluster.sync();      // no CTA may retire while another can still read its shared memory
+    solve_c();
 }
 
 // 4-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros without reading.
