@@ -675,6 +675,14 @@ def run_ours(args, shape):
                                    note="3 fp32 FMA per entry and pending step; peak = measured "
                                         "71.4 TFLOP/s fp32 (nominal 148 SMs x 128 lanes x 1.965 GHz "
                                         "= 74.4)")),
+            steps_kernel=dict(kernel="k_lazy_steps", bound="latency",
+                              launches=phases.get("lazy_steps", (0.0, 0))[1],
+                              ms=phases.get("lazy_steps", (0.0, 0))[0],
+                              us_per_greedy_step=1e3 * phases.get("lazy_steps", (0.0, 0))[0] / max(n_removed, 1),
+                              note="32 sequential greedy steps per launch on a cluster of 4, 2 or 1 CTAs "
+                                   "per layer; a chain of long-latency instructions (cluster barrier, "
+                                   "shuffles, shared-memory loads, float64 conversions), level with the "
+                                   "rank-32 update in summed time but without a throughput roofline"),
             roofline_hessian=dict(
                 kernel="k_row_absmax + k_split_f16 + k_syrk_tc<split>", bound="tensor",
                 achieved=3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0, peak=f16_peak,
