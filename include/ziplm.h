@@ -14,7 +14,11 @@
  *     enqueued there and the stream continues only when it is complete.  Buffers must stay alive
  *     until the stream has drained.  ziplm_prune_layers may run groups of layers concurrently on
  *     up to eight internal non-blocking streams (created once per device, on first use), forked
- *     from and joined back to `cuda_stream` with events.
+ *     from and joined back to `cuda_stream` with events.  Calls on different streams with
+ *     disjoint output and workspace buffers are independent and may overlap on the device
+ *     (inputs may be shared): enqueueing the next batch of layers on a second stream lets its
+ *     tensor-core and float64 phases run under the greedy loop of the first; with several
+ *     batches in flight keep groups x batches at eight or fewer (ZIPLM_OPT_LAYER_GROUPS).
  *   - The return value reports what the host can see when the work is enqueued (bad arguments,
  *     workspace too small, a failed launch).  Failures that depend on the data (a Hessian that
  *     is not positive definite, non-finite values) are written to `layer_status[l]` on the
