@@ -324,6 +324,45 @@ def test_layer_groups_do_not_change_the_result(groups):
         assert torch.equal(ref[k], got[k]), k
 
 
+@pytest.mark.parametrize("groups", [0, 3])
+def test_batches_in_flight_on_two_streams_give_the_results_of_one_at_a_time(groups):
+    """Calls on different streams with their own Hessian, workspace and outputs overlap on the
+    device (the Hessian and inverse of one batch under the loop of the other); every output must
+    be bit-identical to the one the same batch gives on its own."""
+    z = zb()
+    shapes = [wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=320, d_row=48, d_latent=80,
+                        n_tokens=1280, n_layers=6, levels=(256, 100, 0), seed_base=8100 + 50 * b)
+              for b in range(2)]
+    data = [wl.make_layers(sh, "cuda") for sh in shapes]
+    levels = [256, 100, 0]
+    z.set_option(z.Option.LAYER_GROUPS, groups)
+    try:
+        alone = []
+        for W, X in data:
+            H = z.hessian_accumulate(X)
+            alone.append((H, z.prune_layers(W, H, 1, 0.01, levels)))
+            torch.cuda.synchronize()
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        start = torch.cuda.Event()
+        start.record()
+        together = [None, None]
+        for rep in range(2):                       # two rounds, so that calls queue behind calls
+            for b, (W, X) in enumerate(data):
+                with torch.cuda.stream(streams[b]):
+                    streams[b].wait_event(start)
+                    H = z.hessian_accumulate(X)
+                    together[b] = (H, z.prune_layers(W, H, 1, 0.01, levels))
+        torch.cuda.synchronize()
+    finally:
+        z.set_option(z.Option.LAYER_GROUPS, 0)
+    for b in range(2):
+        assert torch.count_nonzero(together[b][1]["layer_status"]) == 0
+        assert torch.equal(alone[b][0], together[b][0])
+        for k in ("order", "W_snap", "loss", "base_loss", "saliency"):
+            assert torch.equal(alone[b][1][k], together[b][1][k]), (b, k)
+    assert not torch.equal(alone[0][1]["order"], alone[1][1]["order"])      # the batches do differ
+
+
 def test_workspace_is_not_assumed_clean(neuron_path):
     """Poison the workspace with NaN bit patterns: values of unused slots never feed live ones."""
     z = zb()
