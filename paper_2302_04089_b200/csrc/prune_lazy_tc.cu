@@ -522,12 +522,16 @@ ziplm_status run_lazy_update_aq_tc(const CUtensorMap& map, const CUtensorMap& ma
     k_lazy_pack_uz<<<dim3(rows_used / 32, L), 256, 0, st>>>(n_pos, m, d, rows_pad, U, Z,
                                                             reinterpret_cast<__nv_bfloat16*>(P));
     ZIPLM_CHECK_LAUNCH();
+    // The kernel is bound by memory bandwidth, which two thirds of the SMs saturate (measured: the
+    // same time with 96 as with 148 CTAs, 12 % more with 74); the others are left to the kernels
+    // of other layer groups and batches that run beside it.
+    const int ctas = (2 * sms + 2) / 3;
     AqSched sch;
     sch.n_strips = rows_used / RM;
     sch.L = L;
     const long long tiles = (long long)L * sch.n_strips * (sch.n_strips + 1) / 2;   // J = 0 .. I
     // about six segments per CTA, so that the last ones to finish differ by a fraction of the run
-    long long seg = tiles / ((long long)sms * 6);
+    long long seg = tiles / ((long long)ctas * 6);
     sch.seg = (int)(seg < 1 ? 1 : (seg > 8 ? 8 : seg));
     sch.prefix[0] = 0;
     for (int k = 0; k < sch.n_strips; ++k) {
@@ -536,7 +540,7 @@ ziplm_status run_lazy_update_aq_tc(const CUtensorMap& map, const CUtensorMap& ma
     }
     for (int k = sch.n_strips + 1; k <= MAX_STRIPS; ++k) sch.prefix[k] = sch.prefix[sch.n_strips];
     sch.n_segments = sch.prefix[sch.n_strips];
-    const int grid = sch.n_segments < sms ? sch.n_segments : sms;
+    const int grid = sch.n_segments < ctas ? sch.n_segments : ctas;
     k_lazy_update_aq_tc<<<grid, AQ_THREADS, AQ_SMEM, st>>>(map, map_a, map_q, sch, n_pos, d, A2, Q2, counter,
                                                           layer_status,
                                                           slot_spin_limit ? slot_spin_limit : kSpinLimit);
