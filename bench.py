@@ -175,10 +175,10 @@ LAZY_REFRESH = 64 # survivors at which that path rebuilds its state exactly (kRe
 # proportion to the layers), not measurements of this run.  Only valid for the bench workload.
 NCU_TRAFFIC = {
     # k_lazy_update_aq_tc, first block at full size (12 layers, 3072 positions of which 3040 live)
-    "k_lazy_update_aq_tc": dict(bytes=3 * (166.8e6 + 249.1e6), launch="n_pos = 3072, m = 32, 12 layers",
+    "k_lazy_update_aq_tc": dict(bytes=3 * (167.8e6 + 249.8e6), launch="n_pos = 3072, m = 32, 12 layers",
                                 algorithmic=12 * 24.0 * 3040 * 3039 / 2),
     # k_lazy_update_aq, a compaction block near full size (12 layers, n_new = 2944)
-    "k_lazy_update_aq": dict(bytes=3 * (162.5e6 + 217.5e6), launch="n_new = 2944, m = 32, 12 layers",
+    "k_lazy_update_aq": dict(bytes=3 * (162.2e6 + 217.4e6), launch="n_new = 2944, m = 32, 12 layers",
                              algorithmic=12 * 24.0 * 2944 * 2943 / 2),
     # k_dgemm_tiles, top-level product F21 = A21 M11^T
     "k_dgemm_tiles": dict(bytes=3 * (116.6e6 + 49.0e6), launch="F21 = A21 M11^T, 12 x 24 macro tiles",
@@ -290,7 +290,9 @@ def run_ours(args, shape):
     # shared): its tensor-core and float64 phases then run under the bandwidth- and latency-bound
     # greedy loop of batch k.  Every step still computes everything; the timed region holds
     # exactly `steps` whole steps between two barriers.
-    B = max(1, args.batches_in_flight)
+    B = args.batches_in_flight
+    if B <= 0:
+        B = 1 if (args.layers or args.max_removed or args.layer_groups) else 2
     groups_per_batch = args.layer_groups if args.layer_groups else (0 if B == 1 else max(1, 6 // B))
     z.set_option(z.Option.LAYER_GROUPS, groups_per_batch)
     slots = [dict(H=H, h_ws=h_ws, p_ws=p_ws, out=out, stream=torch.cuda.Stream() if B > 1 else None)]
@@ -811,9 +813,10 @@ def main():
     ap.add_argument("--compact-every-block", action="store_true",
                     help="delayed-update path: squeeze removed positions out after every block "
                          "(the gathering CUDA-core update only; profiling aid)")
-    ap.add_argument("--batches-in-flight", type=int, default=2,
+    ap.add_argument("--batches-in-flight", type=int, default=0,
                     help="independent batches enqueued concurrently on streams of their own in the "
-                         "timed region (1: one batch at a time)")
+                         "timed region (1: one batch at a time; default 2, or 1 together with the "
+                         "profiling aids --layers, --max-removed and --layer-groups)")
     ap.add_argument("--layer-groups", type=int, default=0,
                     help="profiling aid: number of layer groups on internal streams (0 = library default; "
                          "1 runs them back to back, so that a profiler's per-kernel times add up)")
