@@ -347,6 +347,57 @@ __global__ void __launch_bounds__(256) k_split_f16(const float* __restrict__ X, 
     *reinterpret_cast<uint2*>(lo + row * (size_t)np + k) = b.u;
 }
 
+// Both pre-passes in one for rows of at most 256 * 4 * VEC tokens: a CTA keeps its feature row in
+// registers (VEC 16-byte loads per thread, all in flight together), finds the largest magnitude,
+// and writes the two scaled fp16 parts -- X is read once instead of twice.  Values and layout are
+// those of k_row_absmax followed by k_split_f16.
+template <int VEC>
+__global__ void __launch_bounds__(256) k_row_absmax_split(const float* __restrict__ X, long long ldx,
+                                                          long long N, long long np,
+                                                          unsigned* __restrict__ amax,
+                                                          __half* __restrict__ hi, __half* __restrict__ lo) {
+    __shared__ unsigned red[8];
+    __shared__ unsigned row_max;
+    const size_t row = blockIdx.x;
+    const float* src = X + row * (size_t)ldx;
+    float v[VEC][4];
+    unsigned m = 0u;
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        const long long k = ((long long)j * 256 + threadIdx.x) * 4;
+        v[j][0] = v[j][1] = v[j][2] = v[j][3] = 0.f;
+        if (k + 3 < N) {
+            const float4 t = *reinterpret_cast<const float4*>(src + k);
+            v[j][0] = t.x; v[j][1] = t.y; v[j][2] = t.z; v[j][3] = t.w;
+        } else {
+            for (int e = 0; e < 4; ++e) if (k + e < N) v[j][e] = src[k + e];
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) m = max(m, __float_as_uint(v[j][e]) & 0x7fffffffu);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) m = max(m, red[w]);
+        amax[row] = m;
+        row_max = m;
+    }
+    __syncthreads();
+    const float sc = row_scale(row_max, false);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        const long long k = ((long long)j * 256 + threadIdx.x) * 4;
+        if (k >= np) continue;
+        union { uint2 u; __half h[4]; } a, b;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) split_f16x2(v[j][e] * sc, a.h[e], b.h[e]);
+        *reinterpret_cast<uint2*>(hi + row * (size_t)np + k) = a.u;
+        *reinterpret_cast<uint2*>(lo + row * (size_t)np + k) = b.u;
+    }
+}
+
 // Token-major input (one calibration token per row, as a forward pass emits activations):
 // A is [layers, N, lda] with the feature index contiguous.  A 32 x 32 tile goes through shared
 // memory, so the reads run along features and the writes along tokens, both coalesced; the output
@@ -561,17 +612,27 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
                 }
             } else {
                 const float* Xc = static_cast<const float*>(X) + (size_t)l0 * d * ldx;
-                for (size_t r0 = 0; r0 < rows; r0 += (size_t)1 << 30) {
-                    const size_t rn = rows - r0 < ((size_t)1 << 30) ? rows - r0 : ((size_t)1 << 30);
-                    k_row_absmax<<<(unsigned)rn, 256, 0, st>>>(Xc + r0 * ldx, ldx, N, amax + r0);
-                    ZIPLM_CHECK_LAUNCH();
-                }
-                // grid.y is limited to 65535 rows per launch
-                for (size_t r0 = 0; r0 < rows; r0 += 65535) {
-                    const size_t rn = rows - r0 < 65535 ? rows - r0 : 65535;
-                    k_split_f16<<<dim3((unsigned)((np / 4 + 255) / 256), (unsigned)rn), 256, 0, st>>>(
-                        Xc + r0 * ldx, ldx, N, np, rn, amax + r0, hi + r0 * np, lo + r0 * np);
-                    ZIPLM_CHECK_LAUNCH();
+                constexpr int kFusedVec = 16;     // rows of up to 16384 tokens stay in registers
+                if (np <= 256ll * 4 * kFusedVec) {
+                    for (size_t r0 = 0; r0 < rows; r0 += (size_t)1 << 30) {
+                        const size_t rn = rows - r0 < ((size_t)1 << 30) ? rows - r0 : ((size_t)1 << 30);
+                        k_row_absmax_split<kFusedVec><<<(unsigned)rn, 256, 0, st>>>(
+                            Xc + r0 * ldx, ldx, N, np, amax + r0, hi + r0 * np, lo + r0 * np);
+                        ZIPLM_CHECK_LAUNCH();
+                    }
+                } else {
+                    for (size_t r0 = 0; r0 < rows; r0 += (size_t)1 << 30) {
+                        const size_t rn = rows - r0 < ((size_t)1 << 30) ? rows - r0 : ((size_t)1 << 30);
+                        k_row_absmax<<<(unsigned)rn, 256, 0, st>>>(Xc + r0 * ldx, ldx, N, amax + r0);
+                        ZIPLM_CHECK_LAUNCH();
+                    }
+                    // grid.y is limited to 65535 rows per launch
+                    for (size_t r0 = 0; r0 < rows; r0 += 65535) {
+                        const size_t rn = rows - r0 < 65535 ? rows - r0 : 65535;
+                        k_split_f16<<<dim3((unsigned)((np / 4 + 255) / 256), (unsigned)rn), 256, 0, st>>>(
+                            Xc + r0 * ldx, ldx, N, np, rn, amax + r0, hi + r0 * np, lo + r0 * np);
+                        ZIPLM_CHECK_LAUNCH();
+                    }
                 }
             }
             CUtensorMap mh, ml;
