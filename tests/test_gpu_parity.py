@@ -288,6 +288,19 @@ def test_clustered_steps_kernel_full_depth_every_step(d, check, variant):
     print(reports)
 
 
+def test_full_width_every_step_one_layer_of_3072():
+    """The complete order 3072 -> 0 at the width of the BERT-base fc2 layers (few weight rows, so
+    that the oracle's replay stays within minutes): clusters of 4 CTAs with full slices of 768
+    positions, dense and compaction blocks at full width, the exact rebuild at 64 survivors --
+    every pick, every saliency and every level compared."""
+    sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=3072, d_row=64, d_latent=768,
+                   n_tokens=6144, n_layers=2, levels=tuple(range(2560, -1, -512)))
+    out, reports = run_case(sh, check_layers=[1])
+    assert reports[0]["steps"] == 3072
+    assert reports[0]["max_rho_err"] < 2e-5
+    print(reports)
+
+
 def test_neuron_path_is_deterministic(neuron_path):
     z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=256, d_row=64, d_latent=64,
