@@ -612,12 +612,20 @@ ziplm_status run_hessian_tc(float* H, const void* X, ziplm_dtype dt, bool token_
                 }
             } else {
                 const float* Xc = static_cast<const float*>(X) + (size_t)l0 * d * ldx;
-                constexpr int kFusedVec = 16;     // rows of up to 16384 tokens stay in registers
-                if (np <= 256ll * 4 * kFusedVec) {
+                // rows of up to 16384 tokens stay in registers: 1, 4 or 16 quads per thread
+                if (np <= 256ll * 4 * 16) {
                     for (size_t r0 = 0; r0 < rows; r0 += (size_t)1 << 30) {
                         const size_t rn = rows - r0 < ((size_t)1 << 30) ? rows - r0 : ((size_t)1 << 30);
-                        k_row_absmax_split<kFusedVec><<<(unsigned)rn, 256, 0, st>>>(
-                            Xc + r0 * ldx, ldx, N, np, amax + r0, hi + r0 * np, lo + r0 * np);
+                        const float* xs = Xc + r0 * ldx;
+                        if (np <= 256ll * 4)
+                            k_row_absmax_split<1><<<(unsigned)rn, 256, 0, st>>>(xs, ldx, N, np, amax + r0,
+                                                                                hi + r0 * np, lo + r0 * np);
+                        else if (np <= 256ll * 4 * 4)
+                            k_row_absmax_split<4><<<(unsigned)rn, 256, 0, st>>>(xs, ldx, N, np, amax + r0,
+                                                                                hi + r0 * np, lo + r0 * np);
+                        else
+                            k_row_absmax_split<16><<<(unsigned)rn, 256, 0, st>>>(xs, ldx, N, np, amax + r0,
+                                                                                 hi + r0 * np, lo + r0 * np);
                         ZIPLM_CHECK_LAUNCH();
                     }
                 } else {
