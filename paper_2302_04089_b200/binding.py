@@ -260,8 +260,9 @@ def prune_layers(W: torch.Tensor, H: torch.Tensor, group_size: int, damp_frac: f
     """Greedy structured pruning of L same-shape layers; see ziplm_prune_layers in ziplm.h.
 
     Returns a dict of CUDA tensors: W_snap [L, n_levels, r, d], loss [L, n_levels], base_loss [L]
-    (or None), order [L, G] int32, saliency [L, G] (or None), layer_status [L] int32.  Pass ``out``
-    (a dict from an earlier call) and ``workspace`` to reuse the buffers.
+    (or None), order [L, G] int32, saliency [L, G] (or None), layer_status [L] int32, and the
+    workspace that was used.  Pass ``out`` (a dict from an earlier call) to reuse its buffers,
+    the workspace included when it is large enough and none is given.
     """
     lib = load_library()
     _check(W, torch.float32, "W")
@@ -283,7 +284,13 @@ def prune_layers(W: torch.Tensor, H: torch.Tensor, group_size: int, damp_frac: f
             layer_status=torch.empty(L, dtype=torch.int32, device=dev),
         )
     if workspace is None:
-        workspace = _workspace(prune_workspace_bytes(L, r, d, group_size, n_levels), dev)
+        need = prune_workspace_bytes(L, r, d, group_size, n_levels)
+        kept = out.get("workspace")          # the workspace of the call that produced ``out``
+        if kept is not None and kept.device == dev and kept.numel() >= need:
+            workspace = kept
+        else:
+            out["workspace"] = None          # let go of it before a new one is allocated
+            workspace = _workspace(need, dev)
     lv = (ctypes.c_int * max(n_levels, 1))(*levels)
     with torch.cuda.device(dev):
         st = lib.ziplm_prune_layers(W.data_ptr(), H.data_ptr(), L, r, d, group_size, damp_frac, lv,
