@@ -151,12 +151,13 @@ __device__ __forceinline__ float cand_quotient(const Cand& c) {
 // only the lanes within 1e-5 of the fp32 minimum (almost always a single one) go through the exact
 // float64 comparison, so the common case costs one reduction and six 32-bit shuffles instead of
 // five rounds of 64-bit exchanges.
-__device__ __forceinline__ Cand warp_best(const Cand& mine, float r) {
+__device__ __forceinline__ Cand warp_best(const Cand& mine, float r, float* warp_min = nullptr) {
     // warp minimum in one reduction instruction, on keys that order like the floats they encode
     const unsigned bits = __float_as_uint(r);
     const unsigned key = bits ^ ((bits >> 31) ? 0xffffffffu : 0x80000000u);
     const unsigned kmin = __reduce_min_sync(0xffffffffu, key);
     const float rmin = __uint_as_float(kmin ^ ((kmin >> 31) ? 0x80000000u : 0xffffffffu));
+    if (warp_min) *warp_min = rmin;
     const bool near_min = mine.pos >= 0 && (r == rmin || r <= rmin + fabsf(rmin) * 1e-5f);
     unsigned mask = __ballot_sync(0xffffffffu, near_min);
     Cand best;
@@ -205,6 +206,7 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int compact, int d, int G, int r
     float* sU = reinterpret_cast<float*>(dyn_smem4);       // [BMAX][S]
     float* sZ = sU + (size_t)BMAX * S;                     // [BMAX][S]
     __shared__ Cand s_cand[2][CLUSTER_MAX * NW];           // all warps of the cluster, by step parity
+    __shared__ float s_key[2][CLUSTER_MAX * NW];           // ... and their smallest fp32 quotients
     __shared__ float sT[BMAX][BMAX];                       // T[m][s] = u_s[p_m]
     __shared__ double sTd[BMAX][BMAX];                     // ... in float64, for the solve of c_m
     __shared__ float sUp[BMAX], sZp[BMAX];
@@ -263,18 +265,43 @@ k_lazy_steps(int n0, int S, int t0, int nsteps, int compact, int d, int G, int r
             c.a = da[e]; c.q = dq[e]; c.org = org[e]; c.pos = k0 + e;
             merge_cand(best, c);
         }
-        best = warp_best(best, best.pos >= 0 ? rbest : INFINITY);
+        float wmin;
+        best = warp_best(best, best.pos >= 0 ? rbest : INFINITY, &wmin);
         // push: lane c < CS hands the warp's candidate to CTA c, so that after the barrier every
-        // CTA finds all candidates in its own shared memory
-        if (lane < CS) *cluster.map_shared_rank(&s_cand[par][rank * NW + warp], lane) = best;
+        // CTA finds all candidates in its own shared memory -- together with the warp's smallest
+        // fp32 quotient (within 1e-5 of the candidate's own), the key of the coarse ordering below
+        if (lane < CS) {
+            *cluster.map_shared_rank(&s_cand[par][rank * NW + warp], lane) = best;
+            *cluster.map_shared_rank(&s_key[par][rank * NW + warp], lane) = wmin;
+        }
         cluster.sync();
         // ---- warp 0 of every CTA: global pick from all warps of all CTAs, then the pending
         //      vectors' entries at the pivot (from the CTA that owns it)
         if (warp == 0) {
+            // Coarse ordering by the pushed keys: when exactly one of them lies within 4e-5 of the
+            // smallest (the keys are good to 1e-5), its candidate is the pick and is read directly;
+            // otherwise -- near ties, an invalid entry, nothing left -- all candidates go through
+            // the exact comparison.
             Cand g;
-            g.a = 1.0; g.q = 0.0; g.org = 0x7fffffff; g.pos = -1;
-            for (int e = lane; e < CS * NW; e += 32) merge_cand(g, s_cand[par][e]);
-            g = warp_best(g);
+            {
+                const float k0v = (lane < CS * NW) ? s_key[par][lane] : INFINITY;
+                const float k1v = (lane + 32 < CS * NW) ? s_key[par][lane + 32] : INFINITY;
+                const float kl = fminf(k0v, k1v);
+                const unsigned bits = __float_as_uint(kl);
+                const unsigned key = bits ^ ((bits >> 31) ? 0xffffffffu : 0x80000000u);
+                const unsigned kmin = __reduce_min_sync(0xffffffffu, key);
+                const float rmin = __uint_as_float(kmin ^ ((kmin >> 31) ? 0x80000000u : 0xffffffffu));
+                const float thr = rmin + fabsf(rmin) * 4e-5f;
+                const unsigned n0 = __ballot_sync(0xffffffffu, k0v <= thr);
+                const unsigned n1 = __ballot_sync(0xffffffffu, k1v <= thr);
+                if (fabsf(rmin) < INFINITY && __popc(n0) + __popc(n1) == 1) {
+                    g = s_cand[par][n0 ? __ffs(n0) - 1 : 32 + __ffs(n1) - 1];
+                } else {
+                    g.a = 1.0; g.q = 0.0; g.org = 0x7fffffff; g.pos = -1;
+                    for (int e = lane; e < CS * NW; e += 32) merge_cand(g, s_cand[par][e]);
+                    g = warp_best(g);
+                }
+            }
             int p = g.pos;
             if (p < 0) p = 0;
             double h = g.a;
