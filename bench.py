@@ -743,8 +743,8 @@ def run_ours(args, shape):
                               us_per_greedy_step=1e3 * phases.get("lazy_steps", (0.0, 0))[0] / max(n_removed, 1),
                               note="32 sequential greedy steps per launch on a cluster of 4, 2 or 1 CTAs "
                                    "per layer; a chain of long-latency instructions (cluster barrier, "
-                                   "shuffles, shared-memory loads, float64 conversions), level with the "
-                                   "rank-32 update in summed time but without a throughput roofline"),
+                                   "shuffles, shared-memory loads, float64 conversions), second to the "
+                                   "rank-32 update in summed time and without a throughput roofline"),
             roofline_hessian=dict(
                 kernel="k_row_absmax + k_split_f16 + k_syrk_tc<split>", bound="tensor",
                 achieved=3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0, peak=f16_peak,
