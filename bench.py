@@ -746,7 +746,7 @@ def run_ours(args, shape):
                                    "shuffles, shared-memory loads, float64 conversions), second to the "
                                    "rank-32 update in summed time and without a throughput roofline"),
             roofline_hessian=dict(
-                kernel="k_row_absmax + k_split_f16 + k_syrk_tc<split>", bound="tensor",
+                kernel="k_row_absmax_split + k_syrk_tc<split>", bound="tensor",
                 achieved=3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0, peak=f16_peak,
                 unit="TFLOP/s", frac=(3.0 * hs_useful / (hs_ms * 1e-3) / 1e12 / f16_peak) if hs_ms > 0 else 0.0,
                 useful_tflops=hs_useful / (hs_ms * 1e-3) / 1e12 if hs_ms > 0 else 0.0,
@@ -758,7 +758,7 @@ def run_ours(args, shape):
                 note="fp32 activations: every feature row is scaled by a power of two and split "
                      "into two fp16 parts, every product is three fp16 MMAs (x1*x1, x1*x2, x2*x1), "
                      "so the tensor-pipe work is 3 x the useful d^2 N flop per layer; the time is "
-                     "that of the whole call, the row-maximum and split pre-passes included; the "
+                     "that of the whole call, the row-maximum and split pre-pass included; the "
                      "kernel is bound by its L2 -> shared-memory operand traffic (64 KB per K "
                      "block of 64 tokens against 816 clocks of MMAs)"),
             roofline_streaming_update=dict(
