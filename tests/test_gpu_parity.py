@@ -301,6 +301,19 @@ def test_full_width_every_step_one_layer_of_3072():
     print(reports)
 
 
+def test_cluster_of_eight_every_step_down_to_3072():
+    """Width 4096 (the BERT-large fc2 layers): the steps kernel runs on clusters of 8 CTAs while
+    more than 3072 positions are live, with 64 candidates per pick.  The first 1024 picks, their
+    saliencies and the two levels are compared one by one (few weight rows, so that the oracle's
+    replay stays within two minutes)."""
+    sh = wl.scaled(wl.CONFIGS["c4_bert_large"][1], d_col=4096, d_row=64, d_latent=1024,
+                   n_tokens=8192, n_layers=2, levels=(3584, 3072))
+    out, reports = run_case(sh, check_layers=[0])
+    assert reports[0]["steps"] == 1024
+    assert reports[0]["max_rho_err"] < 2e-5
+    print(reports)
+
+
 def test_neuron_path_is_deterministic(neuron_path):
     z = zb()
     sh = wl.scaled(wl.CONFIGS["c3_bert_base_fc2"][0], d_col=256, d_row=64, d_latent=64,
