@@ -1,10 +1,13 @@
-// Rank-32 update of H^-1 and of the Gram matrix Q = W^T W (delayed Eq. 4 / Eq. 3) for the blocks
-// that leave the removed positions in place, on the 5th-generation tensor cores, as one
-// persistent kernel:
+// Rank-32 update of H^-1, of the Gram matrix Q = W^T W and of W^T itself (delayed Eq. 4 / Eq. 3)
+// for the blocks that leave the removed positions in place, on the 5th-generation tensor cores,
+// as one persistent kernel:
 //
 //   A'[i,j] = A[i,j] - sum_s U[s,i] U[s,j]
 //   Q'[i,j] = Q[i,j] - sum_s (Z[s,i] U[s,j] + U[s,i] Z[s,j]),       i > j positions of the arrays
+//   Wt'[i,c] = Wt[i,c] - sum_s U[s,i] C[s,c],                         c row indices of W
 //
+// (the tiles of W^T follow the tiles of their row strip: the same packed rows of U, the packed C
+// in the place of the column operand, one accumulator, no mirrored store)
 // (the pending vectors are zero at removed positions, whose rows and columns are carried along
 // unchanged).  Nothing is gathered: tiles are plain rectangles, read by TMA and written densely.
 // A pre-pass (k_lazy_pack_uz) transposes the pending vectors to K-major ([position][step]), each
@@ -21,7 +24,7 @@
 //               loads the tile's packed operands by TMA (the 128 rows once per segment, the 128
 //               columns per tile);
 //   warp 1      one thread issues the 36 tcgen05.mma (kind::f16, bfloat16, M = N = 128, K = 16)
-//               of a tile, the smallest partial products first, so that the truncating
+//               of a tile (12 for a tile of W^T), the smallest partial products first, so that the truncating
 //               accumulation meets them while the accumulator is small, into one of two
 //               accumulator stages in tensor memory;
 //   warps 2-17  each owns 32 rows x 64 columns of one matrix (H^-1 or Q) in every tile, worked
@@ -63,12 +66,14 @@ constexpr int AQ_THREADS = 32 * (2 + N_EPI);
 constexpr uint32_t AQ_TMEM_COLS = 512;       // two stages of (H^-1: 128 columns, Q: 128 columns)
 constexpr int DESC_RING = 4;
 constexpr int MAX_STRIPS = 48;               // d <= 6144
-enum { TILE_STOP = 1, TILE_NEW_ROWS = 2 };
+enum { TILE_STOP = 1, TILE_NEW_ROWS = 2, TILE_W = 4 };
 
 // Work list of one launch: the row strips from the longest to the shortest; prefix[k] = number
 // of segments (over all layers) of the k longest strips.
 struct AqSched {
     int n_strips, seg, n_segments, L;
+    int n_wt;                 // tiles of 128 columns of W^T that follow the tiles of a row strip
+    int rows_pad;             // first row of the packed C in P
     int prefix[MAX_STRIPS + 1];
 };
 
@@ -88,13 +93,43 @@ __device__ __forceinline__ void split_bf16x3(float x, __nv_bfloat16 (&p)[3]) {
 // P[l][a][i][64] (bfloat16), a = 0: [U1 | U2], 1: [U3 | Z3], 2: [Z1 | Z2], each half the 32 steps
 // of one part: pending vectors by position, zero for steps >= m and for rows n_pos .. the next
 // multiple of 128.
-__global__ void __launch_bounds__(256) k_lazy_pack_uz(int n_pos, int m, int d, int rows_pad,
+__global__ void __launch_bounds__(256) k_lazy_pack_uz(int n_pos, int m, int d, int rows_pad, int rows_tot,
+                                                      int pos_blocks, int rp,
                                                       const float* __restrict__ U,
                                                       const float* __restrict__ Z,
+                                                      const float* __restrict__ C,
                                                       __nv_bfloat16* __restrict__ P) {
     __shared__ float tu[PK][33], tz[PK][33];
-    const int l = blockIdx.y, i0 = blockIdx.x * 32;
+    const int l = blockIdx.y;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const size_t arr = (size_t)rows_tot * 2 * PK;
+    __nv_bfloat16* Pl = P + (size_t)l * NARR * arr;
+    if ((int)blockIdx.x >= pos_blocks) {
+        // rows rows_pad + c: the scaled pivot columns C[s][c] of W (the column operand of the
+        // tiles of W^T) in the place of U, zeros in the place of Z
+        const int c0 = ((int)blockIdx.x - pos_blocks) * 32;
+        const float* Cl = C + (size_t)l * PK * rp;
+#pragma unroll
+        for (int s = ty; s < PK; s += 8) {
+            const int c = c0 + tx;
+            tu[s][tx] = (c < rp && s < m) ? Cl[(size_t)s * rp + c] : 0.f;
+        }
+        __syncthreads();
+        const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+#pragma unroll
+        for (int rr = ty; rr < 32; rr += 8) {
+            const int i = rows_pad + c0 + rr;
+            if (i >= rows_tot) continue;
+            __nv_bfloat16 u[3];
+            split_bf16x3(tu[tx][rr], u);
+            const size_t o = (size_t)i * 2 * PK + tx;
+            Pl[o] = u[0];            Pl[o + PK] = u[1];
+            Pl[arr + o] = u[2];      Pl[arr + o + PK] = zero;
+            Pl[2 * arr + o] = zero;  Pl[2 * arr + o + PK] = zero;
+        }
+        return;
+    }
+    const int i0 = blockIdx.x * 32;
     const int pos = i0 + tx;
     const int sp = pos < n_pos ? pos : -1;
     const float* Ul = U + (size_t)l * PK * d;
@@ -106,8 +141,6 @@ __global__ void __launch_bounds__(256) k_lazy_pack_uz(int n_pos, int m, int d, i
         tz[s][tx] = ok ? Zl[(size_t)s * d + sp] : 0.f;
     }
     __syncthreads();
-    const size_t arr = (size_t)rows_pad * 2 * PK;
-    __nv_bfloat16* Pl = P + (size_t)l * NARR * arr;
 #pragma unroll
     for (int rr = ty; rr < 32; rr += 8) {
         const int i = i0 + rr;
@@ -124,8 +157,9 @@ __global__ void __launch_bounds__(256) k_lazy_pack_uz(int n_pos, int m, int d, i
 
 __global__ void __launch_bounds__(AQ_THREADS, 1)
 k_lazy_update_aq_tc(const __grid_constant__ CUtensorMap map, const __grid_constant__ CUtensorMap map_a,
-                    const __grid_constant__ CUtensorMap map_q, const __grid_constant__ AqSched sch,
-                    int n_pos, int d, float* __restrict__ A2, float* __restrict__ Q2,
+                    const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_w,
+                    const __grid_constant__ AqSched sch, int n_pos, int d, int rp,
+                    float* __restrict__ A2, float* __restrict__ Q2, float* __restrict__ W2,
                     int* __restrict__ counter, int* __restrict__ layer_status, uint32_t slot_spin_limit) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_tile_full[DESC_RING], bar_tile_empty[DESC_RING];
@@ -185,7 +219,7 @@ k_lazy_update_aq_tc(const __grid_constant__ CUtensorMap map, const __grid_consta
             const int within = s - sch.prefix[k];
             const int segs_strip = (sch.prefix[k + 1] - sch.prefix[k]) / sch.L;
             const int l = within / segs_strip, sidx = within - l * segs_strip;
-            const int nJ = I + 1;                 // tiles J = 0 .. I (the last one holds the diagonal)
+            const int nJ = I + 1 + sch.n_wt;      // tiles J = 0 .. I (the last one holds the diagonal), then W^T
             const int Jb = sidx * sch.seg, Je = min(Jb + sch.seg, nJ);
             const int i0 = I * RM;
             for (int J = Jb; J < Je; ++J, ++t) {
@@ -195,11 +229,13 @@ k_lazy_update_aq_tc(const __grid_constant__ CUtensorMap map, const __grid_consta
                                          mbar_wait_limit(smem_u32(&bar_tile_empty[slot]),
                                                          (uint32_t)(((t >> 2) - 1) & 1), abortp, slot_spin_limit));
                 if (failed) break;
-                const int j0 = J * CN;
+                // a tile of W^T takes its column operand from the rows of P that hold C
+                const bool wtile = J > I;
+                const int j0 = wtile ? sch.rows_pad + (J - I - 1) * CN : J * CN;
                 if (lane == 0) {
                     TileSlot& ts = slots[slot];
                     ts.l = l; ts.i0 = i0; ts.j0 = j0;
-                    ts.flags = (J == Jb) ? TILE_NEW_ROWS : 0;
+                    ts.flags = ((J == Jb) ? TILE_NEW_ROWS : 0) | (wtile ? TILE_W : 0);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_tile_full[slot]));
@@ -280,11 +316,14 @@ k_lazy_update_aq_tc(const __grid_constant__ CUtensorMap map, const __grid_consta
                 // H^-1: U U^T; smallest terms first
                 prod(t_a, U1, U3, true);  prod(t_a, U3, U1, false); prod(t_a, U2, U2, false);
                 prod(t_a, U1, U2, false); prod(t_a, U2, U1, false); prod(t_a, U1, U1, false);
-                // Q: Z U^T + U Z^T
-                prod(t_q, Z1, U3, true);  prod(t_q, Z3, U1, false); prod(t_q, Z2, U2, false);
-                prod(t_q, U1, Z3, false); prod(t_q, U3, Z1, false); prod(t_q, U2, Z2, false);
-                prod(t_q, Z1, U2, false); prod(t_q, Z2, U1, false); prod(t_q, U1, Z2, false);
-                prod(t_q, U2, Z1, false); prod(t_q, Z1, U1, false); prod(t_q, U1, Z1, false);
+                // Q: Z U^T + U Z^T (a tile of W^T has no second matrix: its column operand is C
+                // in the place of U, and the products above are the whole update U^T C)
+                if (!(flags & TILE_W)) {
+                    prod(t_q, Z1, U3, true);  prod(t_q, Z3, U1, false); prod(t_q, Z2, U2, false);
+                    prod(t_q, U1, Z3, false); prod(t_q, U3, Z1, false); prod(t_q, U2, Z2, false);
+                    prod(t_q, Z1, U2, false); prod(t_q, Z2, U1, false); prod(t_q, U1, Z2, false);
+                    prod(t_q, U2, Z1, false); prod(t_q, Z1, U1, false); prod(t_q, U1, Z1, false);
+                }
                 umma_commit(smem_u32(&bar_acc_full[st]));
             }
             if (failed) abort_flag = 1;
@@ -334,8 +373,14 @@ k_lazy_update_aq_tc(const __grid_constant__ CUtensorMap map, const __grid_consta
                 if (lane == 0) {
                     const uint32_t bar = bar0 + 8u * (uint32_t)(c % RING);
                     mbar_expect_tx(bar, (uint32_t)(SLICE_FLOATS * 4));
-                    tma_load_3d(ring_u32 + (uint32_t)((c % RING) * SLICE_FLOATS * 4), min_map, bar,
-                                nj0 + 64 * h + 16 * psub, ni0 + 32 * q, nl);
+                    // a tile of W^T: both matrices' warps bring the same slices in (the second
+                    // copy is served by L2) and work on two of the four each
+                    if (pflags & TILE_W)
+                        tma_load_3d(ring_u32 + (uint32_t)((c % RING) * SLICE_FLOATS * 4), &map_w, bar,
+                                    nj0 - sch.rows_pad + 64 * h + 16 * psub, ni0 + 32 * q, nl);
+                    else
+                        tma_load_3d(ring_u32 + (uint32_t)((c % RING) * SLICE_FLOATS * 4), min_map, bar,
+                                    nj0 + 64 * h + 16 * psub, ni0 + 32 * q, nl);
                 }
                 issued = c + 1;
                 if (++psub == SUBS) {
@@ -366,15 +411,46 @@ k_lazy_update_aq_tc(const __grid_constant__ CUtensorMap map, const __grid_consta
                 if (failed) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 uint32_t v[16];
-                tmem_ld16(lane_taddr + (uint32_t)(stage * 2 * CN + 16 * sub), v);
+                // (a tile of W^T has one accumulator, which both matrices' warps read)
+                tmem_ld16(lane_taddr - ((cflags & TILE_W) ? (uint32_t)(mat * CN) : 0u) +
+                              (uint32_t)(stage * 2 * CN + 16 * sub), v);
                 tmem_ld_wait();
                 if (sub == SUBS - 1) {
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[stage]));
                 }
-                // ---- new entries: old - update, one matrix row per lane
                 float* buf = ring + (size_t)(c % RING) * SLICE_FLOATS;
+                if (cflags & TILE_W) {
+                    // ---- tile of W^T: rows = positions, columns = row indices of W; no mirror.
+                    //      The two warps that share a quarter of the rows and a half of the columns
+                    //      take two of its four slices each.
+                    if ((sub >> 1) == mat) {
+                        float4* b4 = reinterpret_cast<float4*>(buf) + lane * 4;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const int pg = g ^ ((lane >> 1) & 3);
+                            const float4 o = b4[pg];
+                            b4[pg] = make_float4(o.x - __uint_as_float(v[4 * g]), o.y - __uint_as_float(v[4 * g + 1]),
+                                                 o.z - __uint_as_float(v[4 * g + 2]), o.w - __uint_as_float(v[4 * g + 3]));
+                        }
+                        __syncwarp();
+                        float* Wo = W2 + (size_t)cl * d * rp;
+                        const int jc = cj0 - sch.rows_pad + 64 * h + 16 * sub, ib = ci0 + 32 * q;
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) {
+                            const int row = 8 * it + (lane >> 2), u = lane & 3;
+                            const float4 x = reinterpret_cast<const float4*>(buf)[row * 4 + (u ^ ((row >> 1) & 3))];
+                            const int gi = ib + row, gj = jc + 4 * u;
+                            if (gi < n_pos && gj < rp) *reinterpret_cast<float4*>(Wo + (size_t)gi * rp + gj) = x;
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (sub == SUBS - 1) { cl = nl; ci0 = ni0; cj0 = nj0; cflags = pflags; }
+                    continue;
+                }
+                // ---- new entries: old - update, one matrix row per lane
                 float4* b4 = reinterpret_cast<float4*>(buf) + lane * 4;
                 float rr[16];
 #pragma unroll
@@ -470,15 +546,17 @@ int sm_count() {
 }  // namespace
 
 int lazy_tc_rows_pad(int d) { return round_up_int(d, RM); }
+// rows of P: the positions, then the row indices of W (the packed C), both padded to whole tiles
+static int lazy_tc_rows_tot(int d, int rp) { return lazy_tc_rows_pad(d) + round_up_int(rp, CN); }
 
-// size of the packed operands in floats (NARR arrays of 2 * PK bfloat16 per position)
-size_t lazy_tc_pack_floats(int L, int d) { return (size_t)L * NARR * lazy_tc_rows_pad(d) * PK; }
+// size of the packed operands in floats (NARR arrays of 2 * PK bfloat16 per row of P)
+size_t lazy_tc_pack_floats(int L, int d, int rp) { return (size_t)L * NARR * lazy_tc_rows_tot(d, rp) * PK; }
 
-// Tensor map over the packed operands P[L][3][rows_pad][64] (bfloat16): box = 64 rows of one array.
-bool lazy_tc_make_map(CUtensorMap* m, const float* P, int L, int d) {
+// Tensor map over the packed operands P[L][3][rows_tot][64] (bfloat16): box = 64 rows of one array.
+bool lazy_tc_make_map(CUtensorMap* m, const float* P, int L, int d, int rp) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
-    const int rows_pad = lazy_tc_rows_pad(d);
+    const int rows_pad = lazy_tc_rows_tot(d, rp);
     cuuint64_t dims[4] = {(cuuint64_t)2 * PK, (cuuint64_t)rows_pad, NARR, (cuuint64_t)L};
     cuuint64_t strides[3] = {(cuuint64_t)128, (cuuint64_t)rows_pad * 128,
                              (cuuint64_t)NARR * rows_pad * 128};
@@ -489,13 +567,14 @@ bool lazy_tc_make_map(CUtensorMap* m, const float* P, int L, int d) {
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tensor map over one of the fp32 matrices M[L][d][d] (d a multiple of 4): box = 32 rows x 16
-// columns, 64-byte swizzle; what lies outside the matrix reads as zero.
-bool lazy_tc_make_matrix_map(CUtensorMap* m, const float* M, int L, int d) {
+// Tensor map over one of the fp32 matrices M[L][d][cols] (cols a multiple of 4; d for H^-1 and Q,
+// the padded row count of W for W^T): box = 32 rows x 16 columns, 64-byte swizzle; what lies
+// outside the matrix reads as zero.
+bool lazy_tc_make_matrix_map(CUtensorMap* m, const float* M, int L, int d, int cols) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)d, (cuuint64_t)L};
-    cuuint64_t strides[2] = {(cuuint64_t)d * 4, (cuuint64_t)d * d * 4};
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)d, (cuuint64_t)L};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 4, (cuuint64_t)d * cols * 4};
     cuuint32_t box[3] = {16, 32, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(M), dims, strides, box, estr,
@@ -509,18 +588,20 @@ bool lazy_tc_make_matrix_map(CUtensorMap* m, const float* M, int L, int d) {
 // launch; every launch leaves them zero again.  slot_spin_limit = 0 selects the default poll
 // limit of the producer's wait for a free descriptor slot.
 ziplm_status run_lazy_update_aq_tc(const CUtensorMap& map, const CUtensorMap& map_a,
-                                   const CUtensorMap& map_q, int L, int n_pos, int m, int d, float* A2,
-                                   float* Q2, const float* U, const float* Z, float* P, int* counter,
+                                   const CUtensorMap& map_q, const CUtensorMap& map_w, int L, int n_pos,
+                                   int m, int d, int rp, float* A2, float* Q2, float* W2, const float* U,
+                                   const float* Z, const float* C, float* P, int* counter,
                                    int* layer_status, unsigned slot_spin_limit, cudaStream_t st) {
     ZIPLM_CHECK_CUDA(cudaFuncSetAttribute(k_lazy_update_aq_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           AQ_SMEM));
     const int sms = sm_count();
     if (sms <= 0) return ZIPLM_ERR_CUDA;
-    const int rows_pad = lazy_tc_rows_pad(d);
+    const int rows_pad = lazy_tc_rows_pad(d), rows_tot = lazy_tc_rows_tot(d, rp);
     const int rows_used = round_up_int(n_pos, RM);
     if (rows_used / RM > MAX_STRIPS) return ZIPLM_ERR_UNSUPPORTED;
-    k_lazy_pack_uz<<<dim3(rows_used / 32, L), 256, 0, st>>>(n_pos, m, d, rows_pad, U, Z,
-                                                            reinterpret_cast<__nv_bfloat16*>(P));
+    const int pos_blocks = rows_used / 32, c_blocks = (rows_tot - rows_pad) / 32;
+    k_lazy_pack_uz<<<dim3(pos_blocks + c_blocks, L), 256, 0, st>>>(n_pos, m, d, rows_pad, rows_tot, pos_blocks,
+                                                                  rp, U, Z, C, reinterpret_cast<__nv_bfloat16*>(P));
     ZIPLM_CHECK_LAUNCH();
     // The kernel is bound by memory bandwidth, which two thirds of the SMs saturate (measured: the
     // same time with 96 as with 148 CTAs, 12 % more with 74); the others are left to the kernels
@@ -529,20 +610,22 @@ ziplm_status run_lazy_update_aq_tc(const CUtensorMap& map, const CUtensorMap& ma
     AqSched sch;
     sch.n_strips = rows_used / RM;
     sch.L = L;
-    const long long tiles = (long long)L * sch.n_strips * (sch.n_strips + 1) / 2;   // J = 0 .. I
+    sch.n_wt = (rp + CN - 1) / CN;
+    sch.rows_pad = rows_pad;
+    const long long tiles = (long long)L * sch.n_strips * ((sch.n_strips + 1) / 2 + sch.n_wt);   // about
     // about six segments per CTA, so that the last ones to finish differ by a fraction of the run
     long long seg = tiles / ((long long)ctas * 6);
     sch.seg = (int)(seg < 1 ? 1 : (seg > 8 ? 8 : seg));
     sch.prefix[0] = 0;
     for (int k = 0; k < sch.n_strips; ++k) {
-        const int nJ = sch.n_strips - k;          // strip I = n_strips - 1 - k has I + 1 tiles
+        const int nJ = sch.n_strips - k + sch.n_wt;   // strip I = n_strips - 1 - k: I + 1 tiles, then W^T
         sch.prefix[k + 1] = sch.prefix[k] + L * ((nJ + sch.seg - 1) / sch.seg);
     }
     for (int k = sch.n_strips + 1; k <= MAX_STRIPS; ++k) sch.prefix[k] = sch.prefix[sch.n_strips];
     sch.n_segments = sch.prefix[sch.n_strips];
     const int grid = sch.n_segments < ctas ? sch.n_segments : ctas;
-    k_lazy_update_aq_tc<<<grid, AQ_THREADS, AQ_SMEM, st>>>(map, map_a, map_q, sch, n_pos, d, A2, Q2, counter,
-                                                          layer_status,
+    k_lazy_update_aq_tc<<<grid, AQ_THREADS, AQ_SMEM, st>>>(map, map_a, map_q, map_w, sch, n_pos, d, rp, A2, Q2,
+                                                          W2, counter, layer_status,
                                                           slot_spin_limit ? slot_spin_limit : kSpinLimit);
     ZIPLM_CHECK_LAUNCH();
     return ZIPLM_OK;
