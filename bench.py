@@ -169,16 +169,17 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 LAZY_BLOCK = 32   # steps per block of the delayed-update neuron path (BMAX in prune_lazy.cu)
 LAZY_REFRESH = 64 # survivors at which that path rebuilds its state exactly (kRefresh there)
+LAZY_DEAD_MAX, LAZY_DEAD_FRACTION = 128, 16   # its rule for squeezing removed positions out (kDeadMax, kDeadFraction)
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch: constants from earlier
 # ncu captures of these kernels (taken on 4 of the 12 layers and scaled by 3: traffic grows in
 # proportion to the layers), not measurements of this run.  Only valid for the bench workload.
 NCU_TRAFFIC = {
     # k_lazy_update_aq_tc, first block at full size (12 layers, 3072 positions of which 3040 live)
-    "k_lazy_update_aq_tc": dict(bytes=3 * (167.8e6 + 249.8e6), launch="n_pos = 3072, m = 32, 12 layers",
-                                algorithmic=12 * 24.0 * 3040 * 3039 / 2),
+    "k_lazy_update_aq_tc": dict(bytes=3 * (209.6e6 + 291.3e6), launch="n_pos = 3072, m = 32, 12 layers",
+                                algorithmic=12 * (24.0 * 3040 * 3039 / 2 + 8.0 * 768 * 3040)),
     # k_lazy_update_aq, a compaction block near full size (12 layers, n_new = 2944)
-    "k_lazy_update_aq": dict(bytes=3 * (162.2e6 + 217.4e6), launch="n_new = 2944, m = 32, 12 layers",
+    "k_lazy_update_aq": dict(bytes=3 * (162.0e6 + 217.3e6), launch="n_new = 2944, m = 32, 12 layers",
                              algorithmic=12 * 24.0 * 2944 * 2943 / 2),
     # k_dgemm_tiles, top-level product F21 = A21 M11^T
     "k_dgemm_tiles": dict(bytes=3 * (116.6e6 + 49.0e6), launch="F21 = A21 M11^T, 12 x 24 macro tiles",
@@ -189,16 +190,17 @@ NCU_TRAFFIC = {
 }
 
 
-def lazy_update_work(L, G, levels):
+def lazy_update_work(L, G, levels, r=0):
     """Algorithmic work of the rank-32 update of H^-1 and Q (k_lazy_update_aq_tc in blocks that
     leave removed positions in place, k_lazy_update_aq in blocks that squeeze them out) over one
     greedy run: a launch that leaves n live structures reads the off-diagonal entries of H^-1 and
     Q once per symmetric pair and writes them at [i][j] and [j][i] (2 matrices x n(n-1)/2 pairs x
-    4 B x (1 read + 2 writes)) and spends 3 fp32 FMA per pair and pending step.  Rows and columns
-    of removed positions that a dense block still carries are overhead, not counted here.
-    Block boundaries fall on the requested levels, as in the library.  Returns (bytes, fma,
-    launches)."""
-    n, slot, nbytes, fma, launches = G, 0, 0.0, 0.0, 0
+    4 B x (1 read + 2 writes)) and spends 3 fp32 FMA per pair and pending step.  In the dense
+    blocks the same kernel also updates W^T: 8 B x r x n (read + write of the live weights), counted
+    separately.  Rows and columns of removed positions that a dense block still carries are
+    overhead, not counted here.  Block boundaries, and which blocks are dense, as in the library.
+    Returns (bytes, fma, launches, bytes of W^T in the dense blocks)."""
+    n, npos, slot, nbytes, fma, launches, wbytes = G, G, 0, 0.0, 0.0, 0, 0.0
     levels = [v for v in levels if v < G]
     n_min = levels[-1] if levels else G
     while n > n_min:
@@ -206,15 +208,21 @@ def lazy_update_work(L, G, levels):
         if n > LAZY_REFRESH and stop < LAZY_REFRESH:
             stop = LAZY_REFRESH          # the exact rebuild of the state ends a block
         m = min(LAZY_BLOCK, n - stop)
+        dead_after = npos - (n - m)
+        refresh = n > LAZY_REFRESH and n - m == LAZY_REFRESH
+        compact = refresh or dead_after >= LAZY_DEAD_MAX or dead_after * LAZY_DEAD_FRACTION >= npos
         n -= m
+        npos = n if compact else npos
         if n > 1:
             entries = L * n * (n - 1) / 2.0
             nbytes += 24.0 * entries
             fma += 3.0 * m * entries
             launches += 1
+            if not compact:
+                wbytes += 8.0 * L * r * n
         if slot < len(levels) and levels[slot] == n:
             slot += 1
-    return nbytes, fma, launches
+    return nbytes, fma, launches, wbytes
 
 
 def update_bytes(L, r, G, n_removed):
@@ -658,7 +666,8 @@ def run_ours(args, shape):
         prod_tflops = prod_flop / (prod_ms * 1e-3) / 1e12 if prod_ms > 0 else 0.0
         fp64_peak = 37.0      # TFLOP/s, measured with a register-only loop of the float64 mma instruction
         aq_ms, aq_n = phases.get("lazy_update_aq", (0.0, 0))
-        aq_bytes, aq_fma, _ = lazy_update_work(L, G, levels)
+        aq_only_bytes, aq_fma, _, aq_w_bytes = lazy_update_work(L, G, levels, r)
+        aq_bytes = aq_only_bytes + aq_w_bytes
         aq_gbs = aq_bytes / (aq_ms * 1e-3) / 1e9 if aq_ms > 0 else 0.0
         fma_peak = 35.7                                # fp32 TFMA/s measured with a register-only FMA loop
         hs_ms, _ = phases.get("hessian", (0.0, 0))
@@ -716,8 +725,14 @@ def run_ours(args, shape):
                           peak_source=peak_src,
                           launches=aq_n, avg_launch_us=1e3 * aq_ms / max(aq_n, 1),
                           algorithmic_bytes_per_step=aq_bytes,
-                          symmetric=dict(bytes_per_step=aq_bytes * 16.0 / 24.0,
-                                         achieved=aq_gbs * 16.0 / 24.0, frac=aq_gbs * 16.0 / 24.0 / peak,
+                          algorithmic_bytes_note="24 B per symmetric pair of live structures of H^-1 and Q "
+                                                 f"({aq_only_bytes:.4g} B) + 8 B per live weight of W^T in "
+                                                 f"the dense blocks ({aq_w_bytes:.4g} B)",
+                          symmetric=dict(bytes_per_step=aq_only_bytes * 16.0 / 24.0 + aq_w_bytes,
+                                         achieved=(aq_only_bytes * 16.0 / 24.0 + aq_w_bytes) / (aq_ms * 1e-3) / 1e9
+                                         if aq_ms > 0 else 0.0,
+                                         frac=((aq_only_bytes * 16.0 / 24.0 + aq_w_bytes) / (aq_ms * 1e-3) / 1e9 / peak)
+                                         if aq_ms > 0 else 0.0,
                                          note="one read and one write per unique entry of the two "
                                               "symmetric matrices (16 B per pair); the kernel's own "
                                               "count (24 B) includes the second, mirrored store that "
@@ -725,9 +740,10 @@ def run_ours(args, shape):
                           note="rank-32 update of H^-1 and Q, the operation with the largest summed "
                                "time in the timed path (the phase also holds the small kernel that "
                                "packs the pending vectors for the tensor cores).  About three blocks "
-                               "in four leave removed positions in place and run dense 128 x 128 "
-                               "tiles on tcgen05 (bf16 x 3 split of the rank-32 operands, TMA loads, "
-                               "direct and mirrored stores); the others squeeze removed positions "
+                               "in four at full width leave removed positions in place and run dense "
+                               "128 x 128 tiles on tcgen05 (bf16 x 3 split of the rank-32 operands, TMA "
+                               "loads, direct and mirrored stores), W^T included as extra tiles of the "
+                               "same kernel; the others squeeze removed positions "
                                "out with 4-byte gathers on the CUDA cores.  A stand-alone kernel "
                                "with this traffic shape (one read, a direct and a mirrored store per "
                                "entry) and no arithmetic reaches 5.0-5.2 TB/s on this part, 3.3-3.9 "
